@@ -1,0 +1,290 @@
+"""CPU oracle for one step of Efficient Selective Attention (ESA).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+select-plus-attend step computes, written from the paper's equations in numpy
+float64.  It shares no code with the CUDA library and must never be imported
+by it; only the tests, the smoke check and the benchmark's CPU-baseline leg
+call it.
+
+Paper notation: H query heads, H_G key/value heads, d head dim, d_H = H*d,
+d_G = H_G*d, d' = d_c compressed dim; the tokens before the current chunk C
+(t of them) split into initial I, middle M, local L (Section 3.1).
+
+Step, in the paper's order:
+  partition            Section 3.1            I = [0,i_end), M = [i_end,m_end), L = [m_end,t)
+  compress             Eq. 5                  q' = f_q(q), k' = f_k(k): one linear layer each
+  scores               Eq. 6                  S[c,m] = q'_c . k'_m
+  aggregate            Eq. 4                  s_m = max_c ( S[c,m] - max_m' S[c,m'] )
+  proximity_pool       Eq. 8                  s'_j = max of s over [j-eps, j+eps] clipped to M
+  topk                 Eq. 2                  k largest s', ties to the lowest index
+  attend               Eq. 1 / Algorithm 1    softmax attention over I u M_k u L u C (C causal)
+
+Precision (the paper states none; these are the readings the library follows):
+compressor weights are rounded once to bf16; q' and k' are accumulated exactly
+(float64 here) and rounded to bf16; S is rounded to fp32 and Eq. 4 / Eq. 8 run
+in fp32; attention runs in float64 on the bf16 inputs.
+
+Pins (tests/test_oracle_pins.py): attention == textbook causal attention when
+k >= l_M; Algorithm 1's two-part LSE merge == one softmax over the union;
+scores/aggregate/top-k == brute-force loops on tiny inputs; proximity_pool ==
+a library 1-D max pool; compress == plain matrix product and the GQA folding
+identity; the flop/cache closed forms reproduce the paper's 1.56 % and 6.25 %.
+The paper prints no worked numeric example, so absolute output values are
+"parity unpinned" beyond those reductions.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class EsaParams:
+    l_I: int
+    l_L: int
+    k: int
+    eps: int
+    scale: float = 0.0  # softmax scale; 0 -> 1/sqrt(d)
+
+
+# ----------------------------------------------------------------------------
+# rounding helpers
+# ----------------------------------------------------------------------------
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round float64 values to the nearest bf16 value (8 significant bits, ties
+    to even), returned as float64.  Finite, normal-range inputs."""
+    x = np.asarray(x, dtype=np.float64)
+    m, e = np.frexp(x)                      # x = m * 2**e, 0.5 <= |m| < 1
+    return np.ldexp(np.rint(m * 256.0), e - 8)
+
+
+# ----------------------------------------------------------------------------
+# Section 3.1: token partition
+# ----------------------------------------------------------------------------
+def partition(t: int, l_I: int, l_L: int):
+    """Preceding tokens [0,t) -> I=[0,i_end), M=[i_end,m_end), L=[m_end,t).
+    I and L have fixed lengths and are always kept; M is what lies between."""
+    i_end = min(l_I, t)
+    m_end = max(i_end, t - l_L)
+    return i_end, m_end
+
+
+# ----------------------------------------------------------------------------
+# Eq. 5: linear compression of concatenated heads
+# ----------------------------------------------------------------------------
+def compress(X: np.ndarray, W: np.ndarray, b=None) -> np.ndarray:
+    """X [n, d_in] (heads concatenated), W [d', d_in], optional bias [d'] ->
+    bf16-rounded [n, d'].  W is expected already rounded to bf16."""
+    Y = np.asarray(X, np.float64) @ np.asarray(W, np.float64).T
+    if b is not None:
+        Y = Y + np.asarray(b, np.float64)[None, :]
+    return bf16_round(Y)
+
+
+def fold_gqa(W_full: np.ndarray, H: int, H_G: int, d: int) -> np.ndarray:
+    """A [d', H*d] key compressor acting on keys whose H_G heads are repeated
+    H/H_G times equals a [d', H_G*d] compressor with each group's columns
+    summed."""
+    dp = W_full.shape[0]
+    g = H // H_G
+    return np.asarray(W_full, np.float64).reshape(dp, H_G, g, d).sum(axis=2).reshape(dp, H_G * d)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 6, Eq. 4, Eq. 8, Eq. 2
+# ----------------------------------------------------------------------------
+def scores(qc: np.ndarray, kc_M: np.ndarray) -> np.ndarray:
+    """Eq. 6: S[c,m] = q'_c . k'_m  -> fp32 [l_C, l_M]."""
+    return (np.asarray(qc, np.float64) @ np.asarray(kc_M, np.float64).T).astype(np.float32)
+
+
+def aggregate(S: np.ndarray) -> np.ndarray:
+    """Eq. 4 in fp32: s_m = max_c ( S[c,m] - max_{m'} S[c,m'] )."""
+    S = np.asarray(S, np.float32)
+    r = S.max(axis=1, keepdims=True)
+    s = (S - r).max(axis=0)
+    return s + np.float32(0.0)              # -0 -> +0
+
+
+def proximity_pool(s: np.ndarray, eps: int) -> np.ndarray:
+    """Eq. 8: s'_j = max_{w = max(j-eps, first)}^{min(j+eps, last)} s_w, the
+    window clipped to the middle tokens (s covers exactly M)."""
+    s = np.asarray(s, np.float32)
+    n = s.shape[0]
+    out = s.copy()
+    for off in range(1, eps + 1):
+        if off >= n:
+            break
+        out[off:] = np.maximum(out[off:], s[:-off])     # neighbour w = j - off
+        out[:-off] = np.maximum(out[:-off], s[off:])    # neighbour w = j + off
+    return out
+
+
+def topk(sp: np.ndarray, k: int) -> np.ndarray:
+    """Eq. 2: indices (into M) of the k largest scores, larger score first and
+    the lower index first among equal scores; returned in ascending order."""
+    sp = np.asarray(sp, np.float32)
+    k = min(int(k), sp.shape[0])
+    order = np.argsort(-sp, kind="stable")
+    return np.sort(order[:k]).astype(np.int64)
+
+
+def select(qc: np.ndarray, kc_M: np.ndarray, k: int, eps: int):
+    """Scores -> aggregated -> pooled -> top-k.  Returns (indices into M,
+    pooled scores s', row maxima r).  All of M when k >= l_M."""
+    l_M = kc_M.shape[0]
+    if l_M == 0:
+        return np.zeros(0, np.int64), np.zeros(0, np.float32), None
+    S = scores(qc, kc_M)
+    sp = proximity_pool(aggregate(S), eps)
+    if k >= l_M:
+        return np.arange(l_M, dtype=np.int64), sp, S.max(axis=1)
+    return topk(sp, k), sp, S.max(axis=1)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 1 / Algorithm 1: attention over the reduced key set
+# ----------------------------------------------------------------------------
+def attend_positions(t: int, l_C: int, sel_abs: np.ndarray, p: EsaParams) -> np.ndarray:
+    """Key positions attended by the chunk: I, the selected middle tokens, L,
+    then C (C is additionally causal)."""
+    i_end, m_end = partition(t, p.l_I, p.l_L)
+    return np.concatenate([np.arange(0, i_end), np.asarray(sel_abs, np.int64),
+                           np.arange(m_end, t), np.arange(t, t + l_C)]).astype(np.int64)
+
+
+def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t: int,
+           p: EsaParams, return_lse: bool = False):
+    """Eq. 1.  Q_C [l_C,H,d]; K,V [>=t+l_C,H_G,d] with C at [t,t+l_C);
+    sel_abs absolute positions of the selected middle tokens.  Query head h
+    uses key/value head h // (H/H_G).  Query c sees every I, M_k and L key and
+    the C keys at chunk offsets <= c (Algorithm 1: non-causal on [I,M_k],
+    causal with bottom-right alignment on [L,C]).  Returns float64 [l_C,H,d]."""
+    Q_C = np.asarray(Q_C, np.float64)
+    l_C, H, d = Q_C.shape
+    H_G = K.shape[1]
+    g = H // H_G
+    scale = p.scale if p.scale > 0 else 1.0 / np.sqrt(d)
+    pos = attend_positions(t, l_C, sel_abs, p)
+    n_prev = pos.shape[0] - l_C                      # keys before C in the list
+    # visible[c, j]: every key before C; C key u visible iff u <= c
+    visible = np.ones((l_C, pos.shape[0]), dtype=bool)
+    visible[:, n_prev:] = np.tril(np.ones((l_C, l_C), dtype=bool))
+    O = np.empty((l_C, H, d), np.float64)
+    LSE = np.empty((l_C, H), np.float64)
+    for h in range(H):
+        Kh = np.asarray(K[pos, h // g, :], np.float64)
+        Vh = np.asarray(V[pos, h // g, :], np.float64)
+        logits = scale * (Q_C[:, h, :] @ Kh.T)
+        logits = np.where(visible, logits, -np.inf)
+        mx = logits.max(axis=1, keepdims=True)
+        w = np.exp(logits - mx)
+        den = w.sum(axis=1, keepdims=True)
+        O[:, h, :] = (w / den) @ Vh
+        LSE[:, h] = (mx + np.log(den))[:, 0]
+    return (O, LSE) if return_lse else O
+
+
+def _softmax_part(Qh, Kh, Vh, scale, mask):
+    logits = scale * (Qh @ Kh.T)
+    if mask is not None:
+        logits = np.where(mask, logits, -np.inf)
+    mx = logits.max(axis=1, keepdims=True)
+    w = np.exp(logits - mx)
+    den = w.sum(axis=1, keepdims=True)
+    return (w / den) @ Vh, (mx + np.log(den))[:, 0]
+
+
+def attend_alg1(Q_C, K, V, sel_abs, t, p: EsaParams):
+    """Algorithm 1 with identical local and global queries: a causal call on
+    [L,C], a non-causal call on [I,M_k], merged with weights
+    softmax([lse_local, lse_global]) (the exponentials taken after subtracting
+    the larger lse)."""
+    Q_C = np.asarray(Q_C, np.float64)
+    l_C, H, d = Q_C.shape
+    g = H // K.shape[1]
+    scale = p.scale if p.scale > 0 else 1.0 / np.sqrt(d)
+    i_end, m_end = partition(t, p.l_I, p.l_L)
+    gpos = np.concatenate([np.arange(0, i_end), np.asarray(sel_abs, np.int64)]).astype(np.int64)
+    lpos = np.arange(m_end, t + l_C)
+    n_L = t - m_end
+    lmask = np.ones((l_C, lpos.shape[0]), dtype=bool)
+    lmask[:, n_L:] = np.tril(np.ones((l_C, l_C), dtype=bool))
+    O = np.empty((l_C, H, d), np.float64)
+    for h in range(H):
+        Qh = Q_C[:, h, :]
+        l_attn, l_lse = _softmax_part(Qh, np.asarray(K[lpos, h // g], np.float64),
+                                      np.asarray(V[lpos, h // g], np.float64), scale, lmask)
+        if gpos.shape[0] == 0:
+            O[:, h, :] = l_attn
+            continue
+        g_attn, g_lse = _softmax_part(Qh, np.asarray(K[gpos, h // g], np.float64),
+                                      np.asarray(V[gpos, h // g], np.float64), scale, None)
+        top = np.maximum(l_lse, g_lse)
+        se_l, se_g = np.exp(l_lse - top), np.exp(g_lse - top)
+        O[:, h, :] = (l_attn * se_l[:, None] + g_attn * se_g[:, None]) / (se_l + se_g)[:, None]
+    return O
+
+
+# ----------------------------------------------------------------------------
+# one whole step
+# ----------------------------------------------------------------------------
+@dataclass
+class StepResult:
+    sel_abs: np.ndarray     # ascending absolute positions of M_k
+    pooled: np.ndarray      # s' over M (fp32), empty when l_M == 0
+    rowmax: np.ndarray      # r_c (fp32) or None
+    qc: np.ndarray          # compressed queries (bf16 values as float64)
+    O: np.ndarray           # attention output float64 [l_C,H,d]
+    O_bf16: np.ndarray      # the same rounded to bf16 values
+    i_end: int
+    m_end: int
+
+
+def esa_step(Q_C, K, V, Wq, Wk, p: EsaParams, t: int, bq=None, bk=None, Kc=None,
+             do_attend: bool = True) -> StepResult:
+    """One ESA step on a chunk.  Q_C [l_C,H,d]; K,V [>=t+l_C,H_G,d] (bf16 values);
+    Wq [d',d_H], Wk [d',d_G] already rounded to bf16; Kc optionally the cached
+    compressed keys [>=t, d'] (else recomputed from K, of which it is a pure
+    function)."""
+    Q_C = np.asarray(Q_C, np.float64)
+    l_C, H, d = Q_C.shape
+    i_end, m_end = partition(t, p.l_I, p.l_L)
+    qc = compress(Q_C.reshape(l_C, H * d), Wq, bq)
+    if m_end > i_end:
+        if Kc is None:
+            kc_M = compress(np.asarray(K[i_end:m_end], np.float64).reshape(m_end - i_end, -1), Wk, bk)
+        else:
+            kc_M = np.asarray(Kc[i_end:m_end], np.float64)
+        sel, sp, r = select(qc, kc_M, p.k, p.eps)
+        sel_abs = sel + i_end
+    else:
+        sel_abs, sp, r = np.zeros(0, np.int64), np.zeros(0, np.float32), None
+    if do_attend:
+        O = attend(Q_C, K, V, sel_abs, t, p)
+        Ob = bf16_round(O)
+    else:
+        O = Ob = None
+    return StepResult(sel_abs, sp, r, qc, O, Ob, i_end, m_end)
+
+
+# ----------------------------------------------------------------------------
+# Section 3.3 / Appendix A: operation and cache accounting
+# ----------------------------------------------------------------------------
+def flops_full_attention(d_H, H, l_C, l_total):
+    """(4 d_H + 3 H) l_C l_{I,M,L,C}: QK^T, softmax (3 ops per weight), PV."""
+    return (4 * d_H + 3 * H) * l_C * l_total
+
+
+def flops_esa_step(d_H, H, d_c, l_C, l_I, l_M, l_L, k):
+    """Appendix A: compression + selection + sparse attention of one step."""
+    compression = 2 * 2 * l_C * d_H * d_c + 2 * l_C * d_c
+    selection = 2 * l_M * l_C * d_c + l_M * l_C
+    sparse = (4 * d_H + 3 * H) * l_C * (l_I + l_L + l_C + k)
+    return compression, selection, sparse
+
+
+def cache_overhead(d_c, d_G):
+    """Compressed-key cache relative to the K+V cache: d' / (2 d_G)."""
+    return d_c / (2.0 * d_G)
