@@ -1,0 +1,156 @@
+/*
+ * esa.h -- C ABI of the B200 (sm_100a) library for one step of Efficient
+ * Selective Attention (ESA, arXiv 2502.14477).
+ *
+ * One step (Section 3.1 of the paper), for the current chunk C that follows t
+ * cached tokens:
+ *   esa_compress_keys  Eq. 5   k' = f_k(k): compressed keys of C appended to the cache
+ *   esa_select         Eq. 5   q' = f_q(q) for the queries of C
+ *                      Eq. 6   S[c,m] = q'_c . k'_m over the middle tokens M
+ *                      Eq. 4   s_m = max_c ( S[c,m] - max_m' S[c,m'] )
+ *                      Eq. 8   s'_j = max of s over [j-eps, j+eps] clipped to M
+ *                      Eq. 2   the k largest s' (ties: lowest index), ascending positions
+ *   esa_attend         Eq. 1 / Algorithm 1: softmax attention of the queries of C over
+ *                      I u M_k u L u C (C causal), all heads sharing one selection
+ *
+ * Token partition (Section 3.1): with l_I = l_init and l_L = l_local,
+ *   I = [0, i_end), M = [i_end, m_end), L = [m_end, t), C = [t, t + l_C)
+ *   i_end = min(l_I, t), m_end = max(i_end, t - l_L), k_eff = min(top_k, m_end - i_end).
+ *
+ * Conventions
+ *   - Every function returns an esa_status.  Argument, shape and capacity errors are
+ *     found on the host before anything is launched and leave all outputs untouched.
+ *   - "device" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *     ordinary host memory read before the call returns.  The library never frees or
+ *     reallocates caller memory.  Tensors are dense, row-major, bf16 unless noted.
+ *   - *_async variants only enqueue work on the given CUDA stream (a cudaStream_t passed
+ *     as void*) and return without synchronising.  The plain variants run on the legacy
+ *     default stream and return after the work has finished.
+ *   - A context owns device workspace shared by its calls: calls on the same context must
+ *     be ordered (one stream, or externally synchronised).  Use one context per stream.
+ *   - Device-side problems (a bounded wait that ran out) are recorded in a status word
+ *     read by esa_last_device_status; kernels never trap.
+ *   - The compressed-key cache is caller memory with library-defined contents: row p of
+ *     sequence b is k'_p (bf16, d_c values).  n_prev[b] is the only record of its length.
+ */
+#ifndef ESA_H_
+#define ESA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct esa_ctx esa_ctx;
+
+typedef enum {
+    ESA_OK = 0,
+    ESA_ERR_INVALID_ARG = 1,  /* null pointer, negative size, bad handle            */
+    ESA_ERR_SHAPE = 2,        /* a dimension the kernels do not support               */
+    ESA_ERR_CAPACITY = 3,     /* exceeds max_chunk / max_batch / max_tokens           */
+    ESA_ERR_CUDA = 4,         /* a CUDA runtime call failed                           */
+    ESA_ERR_TIMEOUT = 5,      /* a bounded device-side wait ran out                   */
+    ESA_ERR_UNSUPPORTED = 6,  /* valid request the library does not implement         */
+    ESA_ERR_STATE = 7         /* call order: compressors not set                      */
+} esa_status;
+
+/* Hyper-parameters of the step (paper symbols in comments) and capacities. */
+typedef struct {
+    int32_t n_q_heads;     /* H                                                        */
+    int32_t n_kv_heads;    /* H_G, divides H                                           */
+    int32_t head_dim;      /* d: 64 or 128                                             */
+    int32_t d_c;           /* d' : 32, 64 or 128                                       */
+    int32_t l_init;        /* l_I                                                      */
+    int32_t l_local;       /* l_L                                                      */
+    int32_t top_k;         /* k                                                        */
+    int32_t eps;           /* proximity distance of Eq. 8, 0..16                       */
+    int32_t max_chunk;     /* largest l_C of any call                                  */
+    int32_t max_batch;     /* largest B of any call, <= 64                             */
+    int64_t max_tokens;    /* rows per sequence in every cache, < 2^31                 */
+    float softmax_scale;   /* 0 selects 1/sqrt(head_dim)                               */
+} esa_config;
+
+/* Human-readable name of a status code (static storage). */
+const char* esa_status_string(esa_status s);
+
+/* Bytes of device workspace esa_create will allocate for this configuration
+ * (0 if the configuration is invalid). */
+size_t esa_workspace_bytes(const esa_config* cfg);
+
+/* Create a context on the current CUDA device; allocates its workspace there. */
+esa_status esa_create(const esa_config* cfg, esa_ctx** out);
+esa_status esa_destroy(esa_ctx* ctx);
+
+/* Eq. 5: install the two linear compressors.  Host fp32 pointers:
+ * Wq [d_c, H*d], Wk [d_c, H_G*d] (row-major; a key compressor defined on H repeated
+ * heads folds to this shape by summing each group's columns), bq/bk [d_c] or NULL for
+ * no bias.  Weights are rounded once to bf16 (round-to-nearest-even) and copied to
+ * the device; biases stay fp32.  Synchronous. */
+esa_status esa_set_compressors(esa_ctx* ctx, const float* Wq, const float* bq,
+                               const float* Wk, const float* bk);
+
+/* Appends the rows of the current chunk to the caller's K and V caches
+ * (Section 3.1: keys and values of every token are cached; nothing is evicted).
+ * K_new, V_new: device [B, n_new, H_G, d].  K_cache, V_cache: device
+ * [B, max_tokens, H_G, d]; rows [n_prev[b], n_prev[b]+n_new) of sequence b are written.
+ * n_prev: host [B].  ESA_ERR_CAPACITY if n_prev[b]+n_new > max_tokens. */
+esa_status esa_append_kv(esa_ctx* ctx, int32_t B, const void* K_new, const void* V_new,
+                         int32_t n_new, void* K_cache, void* V_cache, const int64_t* n_prev);
+esa_status esa_append_kv_async(esa_ctx* ctx, int32_t B, const void* K_new, const void* V_new,
+                               int32_t n_new, void* K_cache, void* V_cache,
+                               const int64_t* n_prev, void* stream);
+
+/* Eq. 5 for keys: kc_cache[b, n_prev[b] + i, :] = bf16( Wk . K_new[b, i, :, :] + bk ),
+ * fp32 accumulation.  K_new: device [B, n_new, H_G, d].  kc_cache: device
+ * [B, max_tokens, d_c].  n_prev: host [B].  n_new <= max(max_chunk, 4096) per call. */
+esa_status esa_compress_keys(esa_ctx* ctx, int32_t B, const void* K_new, int32_t n_new,
+                             void* kc_cache, const int64_t* n_prev);
+esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, int32_t n_new,
+                                   void* kc_cache, const int64_t* n_prev, void* stream);
+
+/* Eq. 5 (queries), Eq. 6, Eq. 4, Eq. 8, Eq. 2.  Q_cur: device [B, l_C, H, d].
+ * kc_cache must hold k' for positions [0, n_prev[b]) (only M is read).
+ * Outputs: idx_out device int32 [B, top_k]: the first n_sel_out[b] entries of row b are
+ * the selected absolute positions, ascending; n_sel_out device int32 [B] = k_eff.
+ * When k_eff equals the number of middle tokens all of M is returned without scoring.
+ * Scores are fp32; q' is rounded to bf16 like k'. */
+esa_status esa_select(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C,
+                      const void* kc_cache, const int64_t* n_prev,
+                      int32_t* idx_out, int32_t* n_sel_out);
+esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C,
+                            const void* kc_cache, const int64_t* n_prev,
+                            int32_t* idx_out, int32_t* n_sel_out, void* stream);
+
+/* Eq. 1 / Algorithm 1.  Q_cur: device [B, l_C, H, d].  K_cache, V_cache: device
+ * [B, max_tokens, H_G, d] that already hold C at rows [n_prev[b], n_prev[b]+l_C).
+ * idx: device int32 [B, top_k] and n_sel: device int32 [B] as written by esa_select
+ * (positions must lie in M, ascending order is not required).  O: device [B, l_C, H, d]
+ * bf16.  Query head h reads key/value head h / (H/H_G).  Query c of the chunk attends
+ * every I, selected-M and L key and the keys of C at chunk offsets <= c; bf16 products,
+ * fp32 softmax and accumulation. */
+esa_status esa_attend(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C,
+                      const void* K_cache, const void* V_cache, const int64_t* n_prev,
+                      const int32_t* idx, const int32_t* n_sel, void* O);
+esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C,
+                            const void* K_cache, const void* V_cache, const int64_t* n_prev,
+                            const int32_t* idx, const int32_t* n_sel, void* O, void* stream);
+
+/* Diagnostic: copies the pooled scores s' (Eq. 8) of the most recent esa_select of
+ * sequence b to host memory dst[0..n) as fp32, n <= number of middle tokens of that
+ * call.  Synchronises the given stream.  ESA_ERR_STATE if that call did no scoring. */
+esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int64_t n,
+                                  void* stream);
+
+/* Number of kernels this context has launched since creation (host counter). */
+int64_t esa_launch_count(const esa_ctx* ctx);
+
+/* Synchronises the stream, then returns ESA_OK or the error a kernel recorded
+ * (and clears the record). */
+esa_status esa_last_device_status(esa_ctx* ctx, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESA_H_ */

@@ -155,12 +155,13 @@ def attend_positions(t: int, l_C: int, sel_abs: np.ndarray, p: EsaParams) -> np.
 
 
 def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t: int,
-           p: EsaParams, return_lse: bool = False):
+           p: EsaParams, return_lse: bool = False, heads=None):
     """Eq. 1.  Q_C [l_C,H,d]; K,V [>=t+l_C,H_G,d] with C at [t,t+l_C);
     sel_abs absolute positions of the selected middle tokens.  Query head h
     uses key/value head h // (H/H_G).  Query c sees every I, M_k and L key and
     the C keys at chunk offsets <= c (Algorithm 1: non-causal on [I,M_k],
-    causal with bottom-right alignment on [L,C]).  Returns float64 [l_C,H,d]."""
+    causal with bottom-right alignment on [L,C]).  Returns float64 [l_C,H,d];
+    with ``heads`` given only those query heads are computed (the rest are NaN)."""
     Q_C = np.asarray(Q_C, np.float64)
     l_C, H, d = Q_C.shape
     H_G = K.shape[1]
@@ -171,9 +172,9 @@ def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t
     # visible[c, j]: every key before C; C key u visible iff u <= c
     visible = np.ones((l_C, pos.shape[0]), dtype=bool)
     visible[:, n_prev:] = np.tril(np.ones((l_C, l_C), dtype=bool))
-    O = np.empty((l_C, H, d), np.float64)
-    LSE = np.empty((l_C, H), np.float64)
-    for h in range(H):
+    O = np.full((l_C, H, d), np.nan, np.float64)
+    LSE = np.full((l_C, H), np.nan, np.float64)
+    for h in (range(H) if heads is None else heads):
         Kh = np.asarray(K[pos, h // g, :], np.float64)
         Vh = np.asarray(V[pos, h // g, :], np.float64)
         logits = scale * (Q_C[:, h, :] @ Kh.T)
@@ -243,7 +244,7 @@ class StepResult:
 
 
 def esa_step(Q_C, K, V, Wq, Wk, p: EsaParams, t: int, bq=None, bk=None, Kc=None,
-             do_attend: bool = True) -> StepResult:
+             do_attend: bool = True, heads=None) -> StepResult:
     """One ESA step on a chunk.  Q_C [l_C,H,d]; K,V [>=t+l_C,H_G,d] (bf16 values);
     Wq [d',d_H], Wk [d',d_G] already rounded to bf16; Kc optionally the cached
     compressed keys [>=t, d'] (else recomputed from K, of which it is a pure
@@ -262,7 +263,7 @@ def esa_step(Q_C, K, V, Wq, Wk, p: EsaParams, t: int, bq=None, bk=None, Kc=None,
     else:
         sel_abs, sp, r = np.zeros(0, np.int64), np.zeros(0, np.float32), None
     if do_attend:
-        O = attend(Q_C, K, V, sel_abs, t, p)
+        O = attend(Q_C, K, V, sel_abs, t, p, heads=heads)
         Ob = bf16_round(O)
     else:
         O = Ob = None

@@ -1,0 +1,355 @@
+// C ABI of the ESA library: argument checks, token partition (Section 3.1), workspace
+// and launch sequencing.  All arithmetic of the step runs in the kernels.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "esa_internal.h"
+
+using namespace esa;
+
+namespace {
+
+bool config_ok(const esa_config* c) {
+    if (!c) return false;
+    if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->d_c != 32 && c->d_c != 64 && c->d_c != 128) return false;
+    if (c->l_init < 0 || c->l_local < 0 || c->top_k <= 0 || c->eps < 0 || c->eps > 16) return false;
+    if (c->max_chunk <= 0 || c->max_batch <= 0 || c->max_batch > kMaxBatch) return false;
+    if (c->max_tokens <= 0 || c->max_tokens >= (int64_t(1) << 31)) return false;
+    if ((int64_t)c->n_q_heads * c->head_dim % 64 || (int64_t)c->n_kv_heads * c->head_dim % 64) return false;
+    if (!(c->softmax_scale >= 0.f)) return false;
+    return true;
+}
+
+size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct Layout {
+    size_t wq, wk, bq, bk, qc, part, rkey, skey, pkey, att, status, total;
+    size_t part_elems, att_elems;
+};
+
+Layout make_layout(const esa_config* c) {
+    Layout L;
+    const size_t dH = (size_t)c->n_q_heads * c->head_dim, dG = (size_t)c->n_kv_heads * c->head_dim;
+    const size_t rows_max = (size_t)c->max_batch * (c->max_chunk > kCompressMaxRows ? c->max_chunk : kCompressMaxRows);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+    L.wq = take(2 * c->d_c * dH);
+    L.wk = take(2 * c->d_c * dG);
+    L.bq = take(4 * c->d_c);
+    L.bk = take(4 * c->d_c);
+    L.qc = take(2 * (size_t)c->max_batch * c->max_chunk * c->d_c);
+    // split-K partials: up to 16 splits of the largest compression
+    L.part_elems = (size_t)16 * rows_max * c->d_c;
+    if (L.part_elems > (size_t)64 << 20) L.part_elems = (size_t)64 << 20;   // 256 MB cap
+    if (L.part_elems < rows_max * c->d_c) L.part_elems = rows_max * c->d_c;
+    L.part = take(4 * L.part_elems);
+    L.rkey = take(4 * (size_t)c->max_batch * c->max_chunk);
+    L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
+    L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
+    const size_t G = c->n_q_heads / c->n_kv_heads;
+    size_t rows = (size_t)c->max_chunk * G;
+    if (rows > (size_t)kAttSplitRows) rows = kAttSplitRows;
+    L.att_elems = (size_t)c->max_batch * c->n_kv_heads * kAttMaxSplits * rows * (c->head_dim + 2);
+    L.att = take(4 * L.att_elems);
+    L.status = take(256);
+    L.total = off;
+    return L;
+}
+
+uint16_t f32_to_bf16_rne(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);  // NaN
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+esa_status check_common(esa_ctx* ctx, int32_t B) {
+    if (!ctx) return ESA_ERR_INVALID_ARG;
+    if (B <= 0) return ESA_ERR_INVALID_ARG;
+    if (B > ctx->cfg.max_batch) return ESA_ERR_CAPACITY;
+    return ESA_OK;
+}
+
+// Section 3.1 partition for every sequence of the call.
+esa_status build_meta(const esa_ctx* ctx, int B, const int64_t* n_prev, int64_t n_cur, SeqMeta* m,
+                      int* max_lM) {
+    int mx = 0;
+    for (int b = 0; b < B; ++b) {
+        const int64_t t = n_prev[b];
+        if (t < 0) return ESA_ERR_INVALID_ARG;
+        if (t + n_cur > ctx->cfg.max_tokens) return ESA_ERR_CAPACITY;
+        const int64_t i_end = t < ctx->cfg.l_init ? t : ctx->cfg.l_init;
+        int64_t m_end = t - ctx->cfg.l_local;
+        if (m_end < i_end) m_end = i_end;
+        m->t[b] = (int)t;
+        m->i_end[b] = (int)i_end;
+        m->m_end[b] = (int)m_end;
+        if (m_end - i_end > mx) mx = (int)(m_end - i_end);
+    }
+    for (int b = B; b < kMaxBatch; ++b) m->t[b] = m->i_end[b] = m->m_end[b] = 0;
+    if (max_lM) *max_lM = mx;
+    return ESA_OK;
+}
+
+esa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ESA_OK : ESA_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* esa_status_string(esa_status s) {
+    switch (s) {
+        case ESA_OK: return "ESA_OK";
+        case ESA_ERR_INVALID_ARG: return "ESA_ERR_INVALID_ARG";
+        case ESA_ERR_SHAPE: return "ESA_ERR_SHAPE";
+        case ESA_ERR_CAPACITY: return "ESA_ERR_CAPACITY";
+        case ESA_ERR_CUDA: return "ESA_ERR_CUDA";
+        case ESA_ERR_TIMEOUT: return "ESA_ERR_TIMEOUT";
+        case ESA_ERR_UNSUPPORTED: return "ESA_ERR_UNSUPPORTED";
+        case ESA_ERR_STATE: return "ESA_ERR_STATE";
+    }
+    return "ESA_ERR_UNKNOWN";
+}
+
+size_t esa_workspace_bytes(const esa_config* cfg) {
+    if (!config_ok(cfg)) return 0;
+    return make_layout(cfg).total;
+}
+
+esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
+    if (!out) return ESA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!cfg) return ESA_ERR_INVALID_ARG;
+    if (!config_ok(cfg)) return ESA_ERR_SHAPE;
+    esa_ctx* c = new (std::nothrow) esa_ctx();
+    if (!c) return ESA_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->H = cfg->n_q_heads; c->HG = cfg->n_kv_heads; c->d = cfg->head_dim; c->dc = cfg->d_c;
+    c->dH = c->H * c->d; c->dG = c->HG * c->d; c->G = c->H / c->HG;
+    c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)c->d);
+    c->has_w = c->has_bq = c->has_bk = false;
+    c->launches = 0;
+    c->last_scored = false;
+    if (cudaGetDevice(&c->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
+        delete c;
+        return ESA_ERR_CUDA;
+    }
+    Layout L = make_layout(cfg);
+    char* base = nullptr;
+    if (cudaMalloc(&base, L.total) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return ESA_ERR_CUDA;
+    }
+    c->ws_bytes = L.total;
+    c->base = base;
+    c->Wq = reinterpret_cast<__nv_bfloat16*>(base + L.wq);
+    c->Wk = reinterpret_cast<__nv_bfloat16*>(base + L.wk);
+    c->bq = reinterpret_cast<float*>(base + L.bq);
+    c->bk = reinterpret_cast<float*>(base + L.bk);
+    c->Qc = reinterpret_cast<__nv_bfloat16*>(base + L.qc);
+    c->part = reinterpret_cast<float*>(base + L.part);
+    c->part_elems = L.part_elems;
+    c->rkey = reinterpret_cast<uint32_t*>(base + L.rkey);
+    c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
+    c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
+    c->att_part = reinterpret_cast<float*>(base + L.att);
+    c->att_part_elems = L.att_elems;
+    c->status = reinterpret_cast<int*>(base + L.status);
+    if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
+        cudaFree(base);
+        delete c;
+        return ESA_ERR_CUDA;
+    }
+    *out = c;
+    return ESA_OK;
+}
+
+esa_status esa_destroy(esa_ctx* ctx) {
+    if (!ctx) return ESA_ERR_INVALID_ARG;
+    cudaError_t e = cudaFree(ctx->base);
+    delete ctx;
+    return from_cuda(e);
+}
+
+esa_status esa_set_compressors(esa_ctx* ctx, const float* Wq, const float* bq, const float* Wk,
+                               const float* bk) {
+    if (!ctx || !Wq || !Wk) return ESA_ERR_INVALID_ARG;
+    const size_t nq = (size_t)ctx->dc * ctx->dH, nk = (size_t)ctx->dc * ctx->dG;
+    std::vector<uint16_t> hq(nq), hk(nk);
+    for (size_t i = 0; i < nq; ++i) hq[i] = f32_to_bf16_rne(Wq[i]);
+    for (size_t i = 0; i < nk; ++i) hk[i] = f32_to_bf16_rne(Wk[i]);
+    if (cudaMemcpy(ctx->Wq, hq.data(), nq * 2, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
+    if (cudaMemcpy(ctx->Wk, hk.data(), nk * 2, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
+    ctx->has_bq = bq != nullptr;
+    ctx->has_bk = bk != nullptr;
+    if (bq && cudaMemcpy(ctx->bq, bq, 4 * ctx->dc, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
+    if (bk && cudaMemcpy(ctx->bk, bk, 4 * ctx->dc, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
+    ctx->has_w = true;
+    return ESA_OK;
+}
+
+// ------------------------------------------------------------------ append K/V
+esa_status esa_append_kv_async(esa_ctx* ctx, int32_t B, const void* K_new, const void* V_new, int32_t n_new,
+                               void* K_cache, void* V_cache, const int64_t* n_prev, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!K_new || !V_new || !K_cache || !V_cache || !n_prev || n_new < 0) return ESA_ERR_INVALID_ARG;
+    RowMap map;
+    for (int b = 0; b < B; ++b) {
+        if (n_prev[b] < 0) return ESA_ERR_INVALID_ARG;
+        if (n_prev[b] + n_new > ctx->cfg.max_tokens) return ESA_ERR_CAPACITY;
+        map.row0[b] = (int)n_prev[b];
+    }
+    if (n_new == 0) return ESA_OK;
+    return from_cuda(launch_append_kv(ctx, B, (const __nv_bfloat16*)K_new, (const __nv_bfloat16*)V_new, n_new,
+                                      (__nv_bfloat16*)K_cache, (__nv_bfloat16*)V_cache, map,
+                                      (cudaStream_t)stream));
+}
+
+esa_status esa_append_kv(esa_ctx* ctx, int32_t B, const void* K_new, const void* V_new, int32_t n_new,
+                         void* K_cache, void* V_cache, const int64_t* n_prev) {
+    esa_status s = esa_append_kv_async(ctx, B, K_new, V_new, n_new, K_cache, V_cache, n_prev, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
+// ------------------------------------------------------------- compress keys
+esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, int32_t n_new, void* kc_cache,
+                                   const int64_t* n_prev, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!K_new || !kc_cache || !n_prev || n_new < 0) return ESA_ERR_INVALID_ARG;
+    if (!ctx->has_w) return ESA_ERR_STATE;
+    const int cap = ctx->cfg.max_chunk > kCompressMaxRows ? ctx->cfg.max_chunk : kCompressMaxRows;
+    if (n_new > cap) return ESA_ERR_CAPACITY;
+    RowMap map;
+    for (int b = 0; b < B; ++b) {
+        if (n_prev[b] < 0) return ESA_ERR_INVALID_ARG;
+        if (n_prev[b] + n_new > ctx->cfg.max_tokens) return ESA_ERR_CAPACITY;
+        map.row0[b] = (int)n_prev[b];
+    }
+    if (n_new == 0) return ESA_OK;
+    return from_cuda(launch_compress(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, ctx->Wk,
+                                     ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
+                                     ctx->cfg.max_tokens, map, (cudaStream_t)stream));
+}
+
+esa_status esa_compress_keys(esa_ctx* ctx, int32_t B, const void* K_new, int32_t n_new, void* kc_cache,
+                             const int64_t* n_prev) {
+    esa_status s = esa_compress_keys_async(ctx, B, K_new, n_new, kc_cache, n_prev, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
+// -------------------------------------------------------------------- select
+esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* kc_cache,
+                            const int64_t* n_prev, int32_t* idx_out, int32_t* n_sel_out, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!Q_cur || !kc_cache || !n_prev || !idx_out || !n_sel_out || l_C <= 0) return ESA_ERR_INVALID_ARG;
+    if (l_C > ctx->cfg.max_chunk) return ESA_ERR_CAPACITY;
+    if (!ctx->has_w) return ESA_ERR_STATE;
+    SeqMeta meta;
+    int max_lM = 0;
+    s = build_meta(ctx, B, n_prev, l_C, &meta, &max_lM);
+    if (s != ESA_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    bool any_small = false, any_large = false;
+    for (int b = 0; b < B; ++b) {
+        int lM = meta.m_end[b] - meta.i_end[b];
+        ctx->last_lM[b] = lM;
+        if (lM > ctx->cfg.top_k) any_large = true; else any_small = true;
+    }
+    ctx->last_scored = any_large;
+    cudaError_t e = cudaSuccess;
+    if (any_small) {
+        e = launch_select_all(ctx, B, meta, idx_out, n_sel_out, st);
+        if (e != cudaSuccess) return ESA_ERR_CUDA;
+    }
+    if (!any_large) return ESA_OK;
+    // q' = f_q(q) (Eq. 5)
+    RowMap zero;
+    for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
+    e = launch_compress(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
+                        ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, st);
+    if (e != cudaSuccess) return ESA_ERR_CUDA;
+    // sequences that select everything need no scores: give them an empty middle part
+    SeqMeta smeta = meta;
+    for (int b = 0; b < B; ++b)
+        if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
+    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, st);
+    if (e != cudaSuccess) return ESA_ERR_CUDA;
+    e = launch_select(ctx, B, l_C, smeta, max_lM, idx_out, n_sel_out, st);
+    return from_cuda(e);
+}
+
+esa_status esa_select(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* kc_cache,
+                      const int64_t* n_prev, int32_t* idx_out, int32_t* n_sel_out) {
+    esa_status s = esa_select_async(ctx, B, Q_cur, l_C, kc_cache, n_prev, idx_out, n_sel_out, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
+// -------------------------------------------------------------------- attend
+esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                            const void* V_cache, const int64_t* n_prev, const int32_t* idx,
+                            const int32_t* n_sel, void* O, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!Q_cur || !K_cache || !V_cache || !n_prev || !idx || !n_sel || !O || l_C <= 0) return ESA_ERR_INVALID_ARG;
+    if (l_C > ctx->cfg.max_chunk) return ESA_ERR_CAPACITY;
+    SeqMeta meta;
+    s = build_meta(ctx, B, n_prev, l_C, &meta, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)K_cache,
+                                   (const __nv_bfloat16*)V_cache, meta, idx, n_sel, (__nv_bfloat16*)O,
+                                   (cudaStream_t)stream));
+}
+
+esa_status esa_attend(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                      const void* V_cache, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
+                      void* O) {
+    esa_status s = esa_attend_async(ctx, B, Q_cur, l_C, K_cache, V_cache, n_prev, idx, n_sel, O, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
+// --------------------------------------------------------------- diagnostics
+esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int64_t n, void* stream) {
+    if (!ctx || !dst_host || b < 0 || b >= ctx->cfg.max_batch || n < 0) return ESA_ERR_INVALID_ARG;
+    if (!ctx->last_scored || ctx->last_lM[b] <= ctx->cfg.top_k) return ESA_ERR_STATE;
+    if (n > ctx->last_lM[b]) return ESA_ERR_CAPACITY;
+    if (n == 0) return ESA_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the aggregated-score buffer of this sequence is free again after the selection: stage there
+    float* tmp = reinterpret_cast<float*>(ctx->skey + (int64_t)b * ctx->cfg.max_tokens);
+    if (launch_read_pooled(ctx, b, tmp, n, st) != cudaSuccess) return ESA_ERR_CUDA;
+    if (cudaMemcpyAsync(dst_host, tmp, 4 * (size_t)n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ESA_ERR_CUDA;
+    return from_cuda(cudaStreamSynchronize(st));
+}
+
+int64_t esa_launch_count(const esa_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+esa_status esa_last_device_status(esa_ctx* ctx, void* stream) {
+    if (!ctx) return ESA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int h = 0;
+    if (cudaMemcpyAsync(&h, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ESA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ESA_ERR_CUDA;
+    if (h != 0) {
+        if (cudaMemsetAsync(ctx->status, 0, sizeof(int), st) != cudaSuccess) return ESA_ERR_CUDA;
+        return (esa_status)h;
+    }
+    return ESA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,194 @@
+// Eq. 5: the linear compressors q' = f_q(q), k' = f_k(k) as a split-K bf16 GEMM with fp32
+// accumulation, plus the K/V cache append.
+//
+//   Y[r, j] = bf16( sum_i X[r, i] * W[j, i] + bias[j] )
+//
+// X is [rows, d_in] (heads concatenated, Section 3.1 "Efficient Selection"), W is
+// [d_c, d_in]; both are K-major, so the product is a TN GEMM.  The output is only d_c
+// wide, so a chunk yields very few output tiles; the reduction dimension is therefore
+// split across CTAs, each writing an fp32 partial tile, and a second kernel adds the
+// partials in a fixed order (deterministic), adds the bias and rounds to bf16.
+#include "esa_internal.h"
+
+namespace esa {
+
+constexpr int CP_BM = 64;   // rows per CTA (4 warps x 16)
+constexpr int CP_BK = 64;   // reduction elements per pipeline stage
+constexpr int CP_THREADS = 128;
+
+template <int DC>
+__global__ void __launch_bounds__(CP_THREADS)
+compress_partial_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
+                        float* __restrict__ part, int rows, int d_in, int kslice) {
+    constexpr int CH = CP_BK / 8;  // 16-byte chunks per smem row
+    extern __shared__ uint4 smem[];
+    uint4* sX[2] = {smem, smem + CP_BM * CH};
+    uint4* sW[2] = {smem + 2 * CP_BM * CH, smem + 2 * CP_BM * CH + DC * CH};
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row0 = blockIdx.x * CP_BM;
+    const int split = blockIdx.y;
+    const int k_begin = split * kslice;
+    const int nk = kslice / CP_BK;
+
+    auto load_stage = [&](int st, int kk) {
+        const int kofs = k_begin + kk * CP_BK;
+        for (int i = tid; i < CP_BM * CH; i += CP_THREADS) {
+            int r = i / CH, c = i % CH;
+            int gr = row0 + r;
+            bool ok = gr < rows;
+            const __nv_bfloat16* src = X + (size_t)(ok ? gr : 0) * d_in + kofs + c * 8;
+            cp_async16(&sX[st][swz<CH>(r, c)], src, ok ? 16 : 0);
+        }
+        for (int i = tid; i < DC * CH; i += CP_THREADS) {
+            int r = i / CH, c = i % CH;
+            cp_async16(&sW[st][swz<CH>(r, c)], W + (size_t)r * d_in + kofs + c * 8);
+        }
+        cp_async_commit();
+    };
+
+    float acc[DC / 8][4];
+#pragma unroll
+    for (int i = 0; i < DC / 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    load_stage(0, 0);
+    for (int kk = 0; kk < nk; ++kk) {
+        if (kk + 1 < nk) {
+            load_stage((kk + 1) & 1, kk + 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const uint4* tx = sX[kk & 1];
+        const uint4* tw = sW[kk & 1];
+#pragma unroll
+        for (int ks = 0; ks < CP_BK / 16; ++ks) {
+            uint32_t a[4];
+            load_a_frag<CH>(a, tx, warp * 16, ks * 2, lane);
+#pragma unroll
+            for (int nb = 0; nb < DC / 16; ++nb) {
+                uint32_t b[4];
+                load_b_frag_nk<CH>(b, tw, nb * 16, ks * 2, lane);
+                mma_bf16_16816(acc[2 * nb], a, b[0], b[1]);
+                mma_bf16_16816(acc[2 * nb + 1], a, b[2], b[3]);
+            }
+        }
+        __syncthreads();
+    }
+
+    // fp32 partial tile -> part[split][row][DC]
+    const int r_lo = row0 + warp * 16 + (lane >> 2);
+    float* base = part + (size_t)split * rows * DC;
+#pragma unroll
+    for (int nb = 0; nb < DC / 8; ++nb) {
+        int col = nb * 8 + (lane & 3) * 2;
+        if (r_lo < rows) *reinterpret_cast<float2*>(base + (size_t)r_lo * DC + col) = make_float2(acc[nb][0], acc[nb][1]);
+        if (r_lo + 8 < rows)
+            *reinterpret_cast<float2*>(base + (size_t)(r_lo + 8) * DC + col) = make_float2(acc[nb][2], acc[nb][3]);
+    }
+}
+
+// Adds the split-K partials in split order, adds the bias, rounds to bf16 and writes row
+// i of sequence b to dst row b * seq_stride + row0[b] + i.
+__global__ void compress_finalize_kernel(const float* __restrict__ part, const float* __restrict__ bias,
+                                         __nv_bfloat16* __restrict__ dst, int rows, int rows_per_seq,
+                                         int dc, int nsplit, int64_t seq_stride, RowMap map) {
+    const int per_row = dc / 4;
+    int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= (int64_t)rows * per_row) return;
+    int row = (int)(gid / per_row), c4 = (int)(gid % per_row) * 4;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp = 0; sp < nsplit; ++sp) {
+        float4 v = *reinterpret_cast<const float4*>(part + ((size_t)sp * rows + row) * dc + c4);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if (bias) {
+        s.x += bias[c4]; s.y += bias[c4 + 1]; s.z += bias[c4 + 2]; s.w += bias[c4 + 3];
+    }
+    int b = row / rows_per_seq, i = row % rows_per_seq;
+    __nv_bfloat16* o = dst + ((int64_t)b * seq_stride + map.row0[b] + i) * dc + c4;
+    uint2 pk = make_uint2(pack_bf16(s.x, s.y), pack_bf16(s.z, s.w));
+    *reinterpret_cast<uint2*>(o) = pk;
+}
+
+template <int DC>
+static cudaError_t launch_compress_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_per_seq,
+                                     int d_in, const __nv_bfloat16* W, const float* bias,
+                                     __nv_bfloat16* dst, int64_t seq_stride, const RowMap& map,
+                                     cudaStream_t st) {
+    const int row_tiles = (rows + CP_BM - 1) / CP_BM;
+    const int nk_total = d_in / CP_BK;
+    // split the reduction so that about two CTAs per SM are in flight
+    int nsplit = 1;
+    while (nsplit * 2 <= nk_total && (nk_total % (nsplit * 2)) == 0 &&
+           row_tiles * nsplit * 2 <= 2 * ctx->num_sms &&
+           (size_t)(nsplit * 2) * rows * DC <= ctx->part_elems)
+        nsplit *= 2;
+    if ((size_t)nsplit * rows * DC > ctx->part_elems) return cudaErrorInvalidValue;
+    const int kslice = d_in / nsplit;
+    constexpr int smem = 2 * (CP_BM + DC) * (CP_BK / 8) * 16;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(compress_partial_kernel<DC>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    compress_partial_kernel<DC><<<dim3(row_tiles, nsplit), CP_THREADS, smem, st>>>(X, W, ctx->part, rows,
+                                                                                  d_in, kslice);
+    const int64_t n = (int64_t)rows * (DC / 4);
+    compress_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+        ctx->part, bias, dst, rows, rows_per_seq, DC, nsplit, seq_stride, map);
+    ctx->launches += 2;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
+                            const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
+                            int64_t dst_seq_stride, const RowMap& map, cudaStream_t st) {
+    const int rows = B * rows_per_seq;
+    switch (ctx->dc) {
+        case 32: return launch_compress_t<32>(ctx, X, rows, rows_per_seq, d_in, W, bias, dst, dst_seq_stride, map, st);
+        case 64: return launch_compress_t<64>(ctx, X, rows, rows_per_seq, d_in, W, bias, dst, dst_seq_stride, map, st);
+        case 128: return launch_compress_t<128>(ctx, X, rows, rows_per_seq, d_in, W, bias, dst, dst_seq_stride, map, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// ---------------------------------------------------------------------------
+// K/V cache append: rows of the chunk copied into the caller's caches.
+// ---------------------------------------------------------------------------
+__global__ void append_kv_kernel(const uint4* __restrict__ K_new, const uint4* __restrict__ V_new,
+                                 uint4* __restrict__ K_cache, uint4* __restrict__ V_cache, int n_new,
+                                 int row_chunks, int64_t max_tokens, RowMap map) {
+    const int b = blockIdx.y;
+    const int64_t per_seq = (int64_t)n_new * row_chunks;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < per_seq;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t src = (int64_t)b * per_seq + i;
+        int64_t dst = ((int64_t)b * max_tokens + map.row0[b]) * row_chunks + i;
+        K_cache[dst] = K_new[src];
+        V_cache[dst] = V_new[src];
+    }
+}
+
+cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new, const __nv_bfloat16* V_new,
+                             int n_new, __nv_bfloat16* K_cache, __nv_bfloat16* V_cache,
+                             const RowMap& map, cudaStream_t st) {
+    const int row_chunks = ctx->dG / 8;
+    const int64_t per_seq = (int64_t)n_new * row_chunks;
+    int gx = (int)((per_seq + 255) / 256);
+    if (gx > 4 * ctx->num_sms) gx = 4 * ctx->num_sms;
+    if (gx < 1) gx = 1;
+    append_kv_kernel<<<dim3(gx, B), 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(K_new), reinterpret_cast<const uint4*>(V_new),
+        reinterpret_cast<uint4*>(K_cache), reinterpret_cast<uint4*>(V_cache), n_new, row_chunks,
+        ctx->cfg.max_tokens, map);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace esa

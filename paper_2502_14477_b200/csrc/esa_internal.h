@@ -1,0 +1,83 @@
+// Host-side declarations shared by the translation units of the ESA library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/esa.h"
+#include "esa_common.cuh"
+
+namespace esa {
+
+constexpr int kAttMaxSplits = 64;     // split-KV factor of the attention kernel (small chunks)
+constexpr int kAttSplitRows = 64;     // split-KV is used only when l_C * (H/H_G) <= this
+constexpr int kCompressMaxRows = 4096;
+
+// Destination rows of a compression: row i of sequence b goes to
+// dst[(b * seq_stride + row0[b] + i) * d_c ...].
+struct RowMap {
+    int row0[kMaxBatch];
+};
+
+}  // namespace esa
+
+struct esa_ctx {
+    esa_config cfg;
+    int device;
+    void* base;          // the single device allocation every pointer below points into
+    int num_sms;
+    int H, HG, d, dc, dH, dG, G;
+    float scale;
+    bool has_w, has_bq, has_bk;
+    __nv_bfloat16* Wq;   // [dc, dH]
+    __nv_bfloat16* Wk;   // [dc, dG]
+    float* bq;           // [dc]
+    float* bk;           // [dc]
+    __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
+    float* part;         // split-K partial sums of the compression GEMM
+    size_t part_elems;
+    uint32_t* rkey;      // [max_batch * max_chunk] ordered keys of the row maxima r_c
+    uint32_t* skey;      // [max_batch, max_tokens] aggregated scores (ordered keys), or raw fp32 S (l_C = 1)
+    uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys
+    float* att_part;     // split-KV partial outputs + (m, l)
+    size_t att_part_elems;
+    int* status;         // device status word
+    int64_t launches;
+    int last_lM[esa::kMaxBatch];
+    bool last_scored;
+    size_t ws_bytes;
+};
+
+namespace esa {
+
+// Y[dst rows] = bf16( X[rows, d_in] . W[dc, d_in]^T + bias ), fp32 accumulation, split-K.
+cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
+                            const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
+                            int64_t dst_seq_stride, const RowMap& map, cudaStream_t st);
+
+// Eq. 6 + Eq. 4: fills ctx->skey (and ctx->rkey) for the middle tokens of every sequence.
+cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
+                         const SeqMeta& meta, int max_lM, cudaStream_t st);
+
+// Eq. 8 + Eq. 2 on ctx->skey -> idx_out / n_sel_out.
+cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM,
+                          int32_t* idx_out, int32_t* n_sel_out, cudaStream_t st);
+
+// idx_out[b, 0..l_M) = i_end + 0..l_M-1, n_sel_out[b] = l_M for sequences with l_M <= top_k
+// (only_small = 1) or all sequences (only_small = 0).
+cudaError_t launch_select_all(esa_ctx* ctx, int B, const SeqMeta& meta, int32_t* idx_out,
+                              int32_t* n_sel_out, cudaStream_t st);
+
+cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
+                          const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
+                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
+                          cudaStream_t st);
+
+cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new,
+                             const __nv_bfloat16* V_new, int n_new, __nv_bfloat16* K_cache,
+                             __nv_bfloat16* V_cache, const RowMap& map, cudaStream_t st);
+
+cudaError_t launch_read_pooled(esa_ctx* ctx, int b, float* dst_dev, int64_t n, cudaStream_t st);
+
+}  // namespace esa

@@ -1,0 +1,280 @@
+// Eq. 8 + Eq. 2: proximity max-pooling of the aggregated scores and top-k selection.
+//
+//   s'_j = max_{w = max(j-eps, first)}^{min(j+eps, last)} s_w        (Eq. 8, window clipped to M)
+//   M_k  = the k tokens of M with the largest s'                      (Eq. 2)
+//
+// Ties are the rule, not the exception (each query's arg-max scores exactly 0 and the
+// pooling copies every peak to 2*eps+1 neighbours), so the order is total: larger score
+// first, lower index first among equal scores.  Scores are handled as order-preserving
+// uint32 keys.  One thread-block cluster works on one sequence: every CTA pools its
+// slice of M, then three radix passes (11 + 11 + 10 bits, histograms combined through
+// distributed shared memory) find the k-th largest key T, and an index-ordered
+// compaction emits every key > T plus the first (k - #greater) keys == T, which is
+// exactly "lowest index wins" and leaves the output ascending.
+#include <cooperative_groups.h>
+
+#include "esa_internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace esa {
+
+constexpr int SEL_CLUSTER = 8;
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_BINS = 2048;
+
+struct SelectParams {
+    const uint32_t* skey;   // aggregated keys, or raw fp32 S when raw != 0
+    const uint32_t* rkey;   // [B * l_C] (raw mode reads r of query 0)
+    uint32_t* pkey;         // pooled keys out
+    int32_t* idx_out;       // [B, top_k]
+    int32_t* n_sel_out;     // [B]
+    int64_t max_tokens;
+    int top_k;
+    int eps;
+    int raw;
+    int l_C;
+    SeqMeta meta;
+};
+
+__device__ __forceinline__ uint32_t load_agg_key(const uint32_t* src, int m, int raw, float r0) {
+    uint32_t v = src[m];
+    if (raw) return f32_to_key(__uint_as_float(v) - r0);
+    return v;
+}
+
+__global__ void __cluster_dims__(SEL_CLUSTER, 1, 1) __launch_bounds__(SEL_THREADS)
+select_topk_kernel(SelectParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    __shared__ uint32_t hist[SEL_BINS];
+    __shared__ uint32_t warp_cnt[2][32];
+    __shared__ uint32_t cta_cnt[2];          // (#greater, #equal) in this CTA's slice
+    __shared__ uint32_t sh_prefix, sh_krem;  // valid in rank 0: key prefix found so far, k still to place
+    __shared__ uint32_t scan_tmp[SEL_THREADS / 32];
+
+    const int i_end = p.meta.i_end[b];
+    const int l_M = p.meta.m_end[b] - i_end;
+    const int k = p.top_k;
+    // sequences whose middle part fits in k are emitted whole by another kernel
+    // (uniform over the cluster, so no barrier is left waiting)
+    if (l_M <= k) return;
+
+    const uint32_t* src = p.skey + (int64_t)b * p.max_tokens;
+    uint32_t* pk = p.pkey + (int64_t)b * p.max_tokens;
+    const int raw = p.raw;
+    const float r0 = raw ? key_to_f32(p.rkey[(int64_t)b * p.l_C]) : 0.f;
+
+    // slice of this CTA: whole 32-element rows, contiguous
+    const int rows32 = (l_M + 31) / 32;
+    const int rows_per_cta = (rows32 + SEL_CLUSTER - 1) / SEL_CLUSTER;
+    const int lo = min(l_M, rank * rows_per_cta * 32);
+    const int hi = min(l_M, (rank + 1) * rows_per_cta * 32);
+
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+
+    // ---- pass 0: pool (Eq. 8), store pooled keys, histogram of bits 31..21
+    for (int m = lo + tid; m < hi; m += SEL_THREADS) {
+        uint32_t best = load_agg_key(src, m, raw, r0);
+        for (int o = 1; o <= p.eps; ++o) {
+            if (m - o >= 0) best = max(best, load_agg_key(src, m - o, raw, r0));
+            if (m + o < l_M) best = max(best, load_agg_key(src, m + o, raw, r0));
+        }
+        pk[m] = best;
+        atomicAdd(&hist[best >> 21], 1u);
+    }
+
+    uint32_t prefix = 0, krem = (uint32_t)k;
+    // three digit positions: (shift, bits)
+    const int shifts[3] = {21, 10, 0};
+    const int nbits[3] = {11, 11, 10};
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+        cluster.sync();   // all histograms of this pass complete
+        if (rank == 0) {
+            // combine the cluster's histograms into rank 0's copy
+            const int nb = 1 << nbits[pass];
+            for (int i = tid; i < nb; i += SEL_THREADS) {
+                uint32_t s = hist[i];
+                for (int r = 1; r < SEL_CLUSTER; ++r) s += *cluster.map_shared_rank(&hist[i], r);
+                hist[i] = s;
+            }
+            __syncthreads();
+            // find the bin holding the krem-th largest key: suffix sums from the top bin
+            // each thread owns nb / SEL_THREADS consecutive bins (1 or 2), highest bins first
+            const int per = (nb + SEL_THREADS - 1) / SEL_THREADS;
+            uint32_t mine = 0;
+            for (int j = 0; j < per; ++j) {
+                int bin = nb - 1 - (tid * per + j);
+                if (bin >= 0) mine += hist[bin];
+            }
+            // inclusive scan of "mine" over threads
+            uint32_t incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            if (lane == 31) scan_tmp[warp] = incl;
+            __syncthreads();
+            if (warp == 0) {
+                uint32_t w = scan_tmp[lane];
+                uint32_t wi = w;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+                    if (lane >= o) wi += n;
+                }
+                scan_tmp[lane] = wi - w;   // exclusive warp offsets
+            }
+            __syncthreads();
+            uint32_t before = scan_tmp[warp] + incl - mine;   // keys in bins above this thread's bins
+            if (before < krem && before + mine >= krem) {
+                uint32_t acc = before;
+                for (int j = 0; j < per; ++j) {
+                    int bin = nb - 1 - (tid * per + j);
+                    if (bin < 0) break;
+                    uint32_t c = hist[bin];
+                    if (acc + c >= krem) {
+                        sh_prefix = prefix | ((uint32_t)bin << shifts[pass]);
+                        sh_krem = krem - acc;
+                        break;
+                    }
+                    acc += c;
+                }
+            }
+            __syncthreads();
+        }
+        cluster.sync();   // rank 0 published (prefix, krem)
+        prefix = *cluster.map_shared_rank(&sh_prefix, 0);
+        krem = *cluster.map_shared_rank(&sh_krem, 0);
+        cluster.sync();   // everyone has read before rank 0's histogram is reused
+        if (pass == 2) break;
+        // ---- next pass: histogram of the next digit among keys matching the prefix
+        for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
+        __syncthreads();
+        const int sh = shifts[pass + 1];
+        const uint32_t dmask = (1u << nbits[pass + 1]) - 1u;
+        const int psh = shifts[pass];          // bits above psh (inclusive) are fixed
+        for (int m = lo + tid; m < hi; m += SEL_THREADS) {
+            uint32_t key = pk[m];
+            if ((key >> psh) == (prefix >> psh)) atomicAdd(&hist[(key >> sh) & dmask], 1u);
+        }
+    }
+    const uint32_t T = prefix;   // k-th largest key; krem of the keys equal to T are taken
+
+    // ---- ordered compaction
+    // each warp owns a contiguous run of 32-element rows of the CTA's slice
+    const int cta_rows = (hi - lo + 31) / 32;
+    const int rows_per_warp = (cta_rows + 31) / 32;
+    const int w_lo = min(hi, lo + warp * rows_per_warp * 32);
+    const int w_hi = min(hi, lo + (warp + 1) * rows_per_warp * 32);
+    uint32_t n_gt = 0, n_eq = 0;
+    for (int m = w_lo + lane; m < w_hi; m += 32) {
+        uint32_t key = pk[m];
+        n_gt += key > T;
+        n_eq += key == T;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        n_gt += __shfl_xor_sync(0xffffffffu, n_gt, o);
+        n_eq += __shfl_xor_sync(0xffffffffu, n_eq, o);
+    }
+    if (lane == 0) {
+        warp_cnt[0][warp] = n_gt;
+        warp_cnt[1][warp] = n_eq;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t g = warp_cnt[0][lane], e = warp_cnt[1][lane];
+        uint32_t gi = g, ei = e;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t a = __shfl_up_sync(0xffffffffu, gi, o);
+            uint32_t c = __shfl_up_sync(0xffffffffu, ei, o);
+            if (lane >= o) { gi += a; ei += c; }
+        }
+        warp_cnt[0][lane] = gi - g;     // exclusive offsets inside the CTA
+        warp_cnt[1][lane] = ei - e;
+        if (lane == 31) { cta_cnt[0] = gi; cta_cnt[1] = ei; }
+    }
+    cluster.sync();
+    uint32_t gt_before = warp_cnt[0][warp], eq_before = warp_cnt[1][warp];
+    for (int r = 0; r < rank; ++r) {
+        gt_before += *cluster.map_shared_rank(&cta_cnt[0], r);
+        eq_before += *cluster.map_shared_rank(&cta_cnt[1], r);
+    }
+    int32_t* out = p.idx_out + (int64_t)b * p.top_k;
+    for (int m0 = w_lo; m0 < w_hi; m0 += 32) {
+        int m = m0 + lane;
+        uint32_t key = (m < w_hi) ? pk[m] : 0u;
+        bool gt = (m < w_hi) && key > T;
+        bool eq = (m < w_hi) && key == T;
+        uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+        uint32_t lt_mask = (1u << lane) - 1u;
+        uint32_t my_gt = gt_before + __popc(bg & lt_mask);
+        uint32_t my_eq = eq_before + __popc(be & lt_mask);
+        if (gt || (eq && my_eq < krem)) {
+            uint32_t pos = my_gt + min(my_eq, krem);
+            if (pos < (uint32_t)k) out[pos] = i_end + m;
+        }
+        gt_before += __popc(bg);
+        eq_before += __popc(be);
+    }
+    if (rank == 0 && tid == 0) p.n_sel_out[b] = k;
+    cluster.sync();   // keep every CTA's shared memory alive until remote reads are done
+}
+
+// Sequences whose middle part is not larger than k: every middle token is selected.
+__global__ void select_all_kernel(int32_t* idx_out, int32_t* n_sel_out, int top_k, int only_small,
+                                  SeqMeta meta) {
+    const int b = blockIdx.y;
+    const int i_end = meta.i_end[b];
+    const int l_M = meta.m_end[b] - i_end;
+    if (only_small && l_M > top_k) return;
+    const int n = min(l_M, top_k);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        idx_out[(int64_t)b * top_k + i] = i_end + i;
+    if (blockIdx.x == 0 && threadIdx.x == 0) n_sel_out[b] = n;
+}
+
+__global__ void read_pooled_kernel(const uint32_t* __restrict__ pkey, float* __restrict__ dst, int64_t n) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = key_to_f32(pkey[i]);
+}
+
+cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, int32_t* idx_out,
+                          int32_t* n_sel_out, cudaStream_t st) {
+    (void)max_lM;
+    SelectParams p;
+    p.skey = ctx->skey; p.rkey = ctx->rkey; p.pkey = ctx->pkey;
+    p.idx_out = idx_out; p.n_sel_out = n_sel_out;
+    p.max_tokens = ctx->cfg.max_tokens; p.top_k = ctx->cfg.top_k; p.eps = ctx->cfg.eps;
+    p.raw = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
+    select_topk_kernel<<<dim3(SEL_CLUSTER, B), SEL_THREADS, 0, st>>>(p);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select_all(esa_ctx* ctx, int B, const SeqMeta& meta, int32_t* idx_out,
+                              int32_t* n_sel_out, cudaStream_t st) {
+    int gx = (ctx->cfg.top_k + 255) / 256;
+    if (gx > 64) gx = 64;
+    if (gx < 1) gx = 1;
+    select_all_kernel<<<dim3(gx, B), 256, 0, st>>>(idx_out, n_sel_out, ctx->cfg.top_k, 1, meta);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_read_pooled(esa_ctx* ctx, int b, float* dst_dev, int64_t n, cudaStream_t st) {
+    read_pooled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ctx->pkey + (int64_t)b * ctx->cfg.max_tokens,
+                                                                   dst_dev, n);
+    ctx->launches += 1;
+    return cudaGetLastError();
+}
+
+}  // namespace esa

@@ -1,0 +1,293 @@
+"""GPU-vs-oracle parity of the ESA step, through the C ABI (ctypes binding).
+
+Small cases compare every output element; the full-size workloads compare
+sampled chunks / decode steps (each step is a pure function of its inputs, so a
+chunk can be checked without running the ones before it)."""
+import numpy as np
+import pytest
+import torch
+
+import esa_synth as syn
+from oracle import esa_oracle as orc
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+
+
+def fill_kc_gpu(ctx, seq: hp.DeviceSeq, upto: int, step: int = 4096):
+    """k' for rows [0, upto) of every sequence, by the library itself."""
+    for r0 in range(0, upto, step):
+        r1 = min(upto, r0 + step)
+        ctx.compress_keys(seq.K[:, r0:r1].contiguous(), seq.Kc, [r0] * seq.B)
+
+
+def oracle_kc_bits(cfg, K64: np.ndarray, Wk) -> np.ndarray:
+    kc = orc.compress(K64.reshape(K64.shape[0], -1), Wk)
+    return syn.to_bf16_bits(kc.astype(np.float32))
+
+
+def run_step_gpu(ctx, seq: hp.DeviceSeq, Q: torch.Tensor, t_list, do_compress=True):
+    B, l_C = Q.shape[0], Q.shape[1]
+    if do_compress:
+        Knew = torch.stack([seq.K[b, t_list[b]: t_list[b] + l_C] for b in range(B)]).contiguous()
+        ctx.compress_keys(Knew, seq.Kc, t_list)
+    ctx.select(Q, seq.Kc, t_list, seq.idx, seq.n_sel)
+    O = torch.empty_like(Q)
+    ctx.attend(Q, seq.K, seq.V, t_list, seq.idx, seq.n_sel, O)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    n = seq.n_sel.cpu().numpy()
+    idx = seq.idx.cpu().numpy()
+    return [idx[b, : n[b]].astype(np.int64) for b in range(B)], O
+
+
+# --------------------------------------------------------------- compression
+@pytest.mark.parametrize("name,n_new,with_bias", [("c1", 128, False), ("c1", 37, True), ("c2", 512, False),
+                                                   ("c2", 1, False), ("c2", 700, True)])
+def test_compress_keys_parity(name, n_new, with_bias):
+    cfg = syn.get_config(name).with_(S=2048, n_decode=0)
+    bias = syn.compressor_bias(cfg) if with_bias else None
+    ctx = hp.make_esa(cfg, max_tokens=2048, max_chunk=1024, max_batch=2, bias=bias)
+    _, _, Wq, Wk = hp.oracle_weights(cfg)
+    B = 2
+    n_prev = [5, 1000]
+    Kbits = [syn.qkv_rows(cfg, "k", 0, n_new, 0, b) for b in range(B)]
+    Knew = torch.stack([hp.bits_to_torch(x) for x in Kbits])
+    kc = torch.zeros(B, 2048, cfg.d_c, dtype=torch.bfloat16, device="cuda")
+    ctx.compress_keys(Knew, kc, n_prev, sync=True)
+    for b in range(B):
+        X = syn.bf16_bits_to_f64(Kbits[b]).reshape(n_new, -1)
+        hp.check_compressed(kc[b, n_prev[b]: n_prev[b] + n_new], X, Wk, None if bias is None else bias[1],
+                            what=f"{name} b{b}")
+        # rows outside the appended range stay untouched
+        assert float(kc[b, : n_prev[b]].abs().sum()) == 0.0
+        assert float(kc[b, n_prev[b] + n_new:].abs().sum()) == 0.0
+
+
+def test_append_kv_copies_rows():
+    cfg = syn.get_config("c1").with_(S=512, n_decode=0)
+    ctx = hp.make_esa(cfg, max_tokens=512, max_batch=3)
+    B, n_new = 3, 19
+    Knew = torch.randn(B, n_new, cfg.H_G, cfg.d, device="cuda").bfloat16()
+    Vnew = torch.randn(B, n_new, cfg.H_G, cfg.d, device="cuda").bfloat16()
+    Kc = torch.zeros(B, 512, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    n_prev = [0, 100, 493]
+    ctx.append_kv(Knew, Vnew, Kc, Vc, n_prev, sync=True)
+    for b in range(B):
+        assert torch.equal(Kc[b, n_prev[b]: n_prev[b] + n_new], Knew[b])
+        assert torch.equal(Vc[b, n_prev[b]: n_prev[b] + n_new], Vnew[b])
+        assert float(Kc[b].abs().sum()) == float(Knew[b].abs().sum())
+
+
+# ---------------------------------------------- stage-isolated select / attend
+def _stage_isolated(cfg, t, l_C, layer=0, eps=None, heads=None, check_scores=True):
+    """GPU select fed the ORACLE's compressed keys; GPU attend fed the ORACLE's selection."""
+    eps = cfg.eps if eps is None else eps
+    p = orc.EsaParams(cfg.l_I, cfg.l_L, cfg.k, eps)
+    _, _, Wq, Wk = hp.oracle_weights(cfg, layer)
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=1, layer=layer, eps=eps)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, layer=layer, B=1)
+    seq.fill_kv(0, n)
+    K64 = hp.torch_to_f64(seq.K[0])
+    V64 = hp.torch_to_f64(seq.V[0])
+    Qb = syn.qkv_rows(cfg, "q", t, t + l_C, layer, 0)
+    Q = hp.bits_to_torch(Qb)[None].contiguous()
+    Q64 = syn.bf16_bits_to_f64(Qb)
+    Kc64 = orc.compress(K64.reshape(n, -1), Wk)
+    seq.Kc[0] = hp.bits_to_torch(syn.to_bf16_bits(Kc64.astype(np.float32)))
+    res = orc.esa_step(Q64, K64, V64, Wq, Wk, p, t, Kc=Kc64, heads=heads)
+    # select
+    ctx.select(Q, seq.Kc, [t], seq.idx, seq.n_sel, sync=True)
+    n_sel = int(seq.n_sel[0])
+    sel_gpu = seq.idx[0, :n_sel].cpu().numpy().astype(np.int64)
+    ndiff = hp.check_index_sets(sel_gpu, res, cfg.k, what=f"{cfg.name} t={t}")
+    l_M = res.m_end - res.i_end
+    if check_scores and l_M > cfg.k:
+        sp_gpu = ctx.read_pooled_scores(0, l_M)
+        scale = float(np.max(np.abs(res.rowmax)))
+        err = np.max(np.abs(sp_gpu.astype(np.float64) - res.pooled.astype(np.float64)))
+        assert err <= 2e-3 * scale, f"pooled scores differ by {err} (scale {scale})"
+        assert sp_gpu.max() == 0.0 and np.all(sp_gpu <= 0)
+    # attend on the oracle's selection
+    seq.idx[0, : len(res.sel_abs)] = torch.from_numpy(res.sel_abs.astype(np.int32)).cuda()
+    seq.n_sel[0] = len(res.sel_abs)
+    O = torch.empty_like(Q)
+    ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O, sync=True)
+    hp.check_attention(O[0], res.O, what=f"{cfg.name} t={t}", heads=heads)
+    assert ctx.last_device_status() == 0
+    return ndiff
+
+
+@pytest.mark.parametrize("t,l_C", [(0, 128), (128, 128), (640, 128), (768, 128), (772, 128), (773, 128),
+                                   (1536, 128), (3968, 128), (4000, 77), (4096, 1), (4111, 1), (2000, 5)])
+def test_c1_stage_isolated(t, l_C):
+    _stage_isolated(syn.get_config("c1"), t, l_C)
+
+
+@pytest.mark.parametrize("eps", [0, 1, 5])
+def test_c1_eps_variants(eps):
+    _stage_isolated(syn.get_config("c1"), 3968, 128, eps=eps)
+    _stage_isolated(syn.get_config("c1"), 4100, 1, eps=eps)
+
+
+def test_c2_shape_stage_isolated_mid_chunk():
+    _stage_isolated(syn.get_config("c2"), 16 * 512, 512, heads=[0, 5, 31])
+
+
+def test_gqa_group_of_seven_stage_isolated():
+    cfg = syn.get_config("c4").with_(S=16384, l_C=256, l_L=1024, k=1024)
+    _stage_isolated(cfg, 40 * 256, 256, heads=[0, 6, 7, 27])
+    _stage_isolated(cfg, 10000, 1, heads=None)
+
+
+def test_all_equal_scores_take_lowest_indices():
+    """Identical compressed keys give identical scores: the first k middle tokens win."""
+    cfg = syn.get_config("c1")
+    t, l_C = 2048, 128
+    ctx = hp.make_esa(cfg, max_tokens=t + l_C, max_batch=1)
+    kc = torch.ones(1, t + l_C, cfg.d_c, dtype=torch.bfloat16, device="cuda")
+    Q = hp.bits_to_torch(syn.qkv_rows(cfg, "q", t, t + l_C))[None].contiguous()
+    idx = torch.zeros(1, cfg.k, dtype=torch.int32, device="cuda")
+    n_sel = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.select(Q, kc, [t], idx, n_sel, sync=True)
+    assert int(n_sel[0]) == cfg.k
+    assert idx[0].cpu().tolist() == list(range(cfg.l_I, cfg.l_I + cfg.k))
+
+
+# ------------------------------------------------------ end to end, config 1
+def test_c1_end_to_end_prefill_and_decode():
+    cfg = syn.get_config("c1")
+    p = hp.oracle_params(cfg)
+    _, _, Wq, Wk = hp.oracle_weights(cfg)
+    ctx = hp.make_esa(cfg)
+    seq = hp.DeviceSeq(cfg)
+    n = cfg.max_tokens
+    Kb, Vb = syn.qkv_rows(cfg, "k", 0, n), syn.qkv_rows(cfg, "v", 0, n)
+    K64, V64 = syn.bf16_bits_to_f64(Kb), syn.bf16_bits_to_f64(Vb)
+    Kdev, Vdev = hp.bits_to_torch(Kb), hp.bits_to_torch(Vb)
+    Qb = syn.qkv_rows(cfg, "q", 0, n)
+    steps = [(t, cfg.l_C) for t in range(0, cfg.S, cfg.l_C)] + [(cfg.S + i, 1) for i in range(cfg.n_decode)]
+    total_diff = 0
+    for t, l_C in steps:
+        Knew, Vnew = Kdev[None, t: t + l_C].contiguous(), Vdev[None, t: t + l_C].contiguous()
+        ctx.append_kv(Knew, Vnew, seq.K, seq.V, [t])
+        Q = hp.bits_to_torch(Qb[t: t + l_C])[None].contiguous()
+        sel, O = run_step_gpu(ctx, seq, Q, [t])
+        res = orc.esa_step(syn.bf16_bits_to_f64(Qb[t: t + l_C]), K64[: t + l_C], V64[: t + l_C], Wq, Wk, p, t)
+        total_diff += hp.check_index_sets(sel[0], res, cfg.k, what=f"c1 t={t}")
+        hp.check_attention(O[0], res.O, what=f"c1 t={t}")
+    # the library's own compressed-key cache against the exact product
+    hp.check_compressed(seq.Kc[0, :n], K64.reshape(n, -1), Wk, what="c1 cache")
+    assert total_diff <= 0.01 * cfg.k * len(steps)
+
+
+# --------------------------------------------- full-size workloads, sampled
+def _sampled_prefill(cfg, chunks, layer=0, heads=None):
+    p = hp.oracle_params(cfg)
+    _, _, Wq, Wk = hp.oracle_weights(cfg, layer)
+    t_max = max(chunks) * cfg.l_C
+    n = t_max + cfg.l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_batch=1, layer=layer)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, layer=layer, B=1)
+    seq.fill_kv(0, n)
+    fill_kc_gpu(ctx, seq, n)
+    K64 = hp.torch_to_f64(seq.K[0])
+    V64 = hp.torch_to_f64(seq.V[0])
+    out = []
+    for c in chunks:
+        t = c * cfg.l_C
+        Qb = syn.qkv_rows(cfg, "q", t, t + cfg.l_C, layer, 0)
+        Q = hp.bits_to_torch(Qb)[None].contiguous()
+        sel, O = run_step_gpu(ctx, seq, Q, [t], do_compress=False)
+        res = orc.esa_step(syn.bf16_bits_to_f64(Qb), K64[: t + cfg.l_C], V64[: t + cfg.l_C], Wq, Wk, p, t, heads=heads)
+        nd = hp.check_index_sets(sel[0], res, cfg.k, what=f"{cfg.name} chunk {c}")
+        # attention is compared on the oracle's own selection unless the sets agree exactly
+        if nd:
+            seq.idx[0, : len(res.sel_abs)] = torch.from_numpy(res.sel_abs.astype(np.int32)).cuda()
+            ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O, sync=True)
+        hp.check_attention(O[0], res.O, what=f"{cfg.name} chunk {c}", heads=heads)
+        out.append((sel[0], res))
+    return out
+
+
+def test_c2_sampled_chunks():
+    # first chunk, last chunk without middle tokens, first with l_M > k, a middle one, the last
+    _sampled_prefill(syn.get_config("c2"), [0, 4, 13, 40, 63], heads=[0, 9, 18, 31])
+
+
+def test_c4_sampled_chunks():
+    cfg = syn.get_config("c4")
+    _sampled_prefill(cfg, [5, 13, 255], heads=[0, 13, 27])
+
+
+def test_c5_needle_chunks():
+    cfg = syn.get_config("c5")
+    for layer in (0, 3):
+        plan = syn.needle_plan(cfg, layer)
+        span = int(np.argmax(plan.aligned_chunk))          # the latest aligned chunk of this layer
+        chunk = int(plan.aligned_chunk[span])
+        out = _sampled_prefill(cfg, [chunk], layer=layer, heads=[0, 17])
+        sel, res = out[0]
+        chosen = set(sel.tolist())
+        for i in plan.spans_in_chunk(chunk):
+            for tok in plan.needle_tokens(i):
+                if res.i_end <= tok < res.m_end:
+                    assert tok in chosen, f"needle token {tok} of span {i} not selected"
+
+
+def test_c3_decode_steps():
+    cfg = syn.get_config("c3")
+    p = hp.oracle_params(cfg)
+    _, _, Wq, Wk = hp.oracle_weights(cfg)
+    ctx = hp.make_esa(cfg)
+    seq = hp.DeviceSeq(cfg)
+    n = cfg.max_tokens
+    seq.fill_kv(0, n)
+    fill_kc_gpu(ctx, seq, cfg.S)
+    for step in (0, 1, 127, 255):
+        t = cfg.S + step
+        # k' of the tokens decoded before this step (rows S..t) are appended by the library
+        if step > 0:
+            upto = [cfg.S] * cfg.B
+            ctx.compress_keys(seq.K[:, cfg.S: t].contiguous(), seq.Kc, upto)
+        Q = seq.q_rows(t, t + 1).contiguous()
+        sel, O = run_step_gpu(ctx, seq, Q, [t] * cfg.B)
+        for b in (0, 3, 7) if step else range(cfg.B):
+            K64 = hp.torch_to_f64(seq.K[b, : t + 1])
+            V64 = hp.torch_to_f64(seq.V[b, : t + 1])
+            res = orc.esa_step(hp.torch_to_f64(Q[b]), K64, V64, Wq, Wk, p, t)
+            nd = hp.check_index_sets(sel[b], res, cfg.k, what=f"c3 step {step} seq {b}")
+            if nd == 0:
+                hp.check_attention(O[b], res.O, what=f"c3 step {step} seq {b}")
+
+
+# ----------------------------------------------------------------- error paths
+def test_argument_errors_leave_outputs_untouched():
+    import paper_2502_14477_b200 as esa
+    cfg = syn.get_config("c1")
+    ctx = hp.make_esa(cfg, max_tokens=1024, max_batch=1)
+    Q = torch.zeros(1, 128, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda")
+    kc = torch.zeros(1, 1024, cfg.d_c, dtype=torch.bfloat16, device="cuda")
+    idx = torch.full((1, cfg.k), -7, dtype=torch.int32, device="cuda")
+    n_sel = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    with pytest.raises(esa.EsaError) as e:
+        ctx.select(Q, kc, [1000], idx, n_sel, sync=True)          # 1000 + 128 > max_tokens
+    assert e.value.status == 3
+    with pytest.raises(esa.EsaError) as e:
+        ctx.select(Q, kc, [-1], idx, n_sel, sync=True)
+    assert e.value.status == 1
+    assert int(idx.min()) == -7 and int(n_sel[0]) == -7
+    ctx2 = esa.Esa(esa.EsaConfig(cfg.H, cfg.H_G, cfg.d, cfg.d_c, 4, 512, 256, 3, 128, 1, 1024))
+    with pytest.raises(esa.EsaError) as e:
+        ctx2.select(Q, kc, [0], idx, n_sel, sync=True)            # compressors not set
+    assert e.value.status == 7
+    with pytest.raises(esa.EsaError):
+        esa.Esa(esa.EsaConfig(7, 2, 64, 32, 4, 512, 256, 3, 128, 1, 1024))   # H not a multiple of H_G
