@@ -1,0 +1,475 @@
+#!/usr/bin/env python
+"""Benchmark of the ESA select-plus-attend step on B200.
+
+Headline workload (config "c5" shape): one layer of the Llama-3-8B attention
+shape (H=32, H_G=8, d=128, d'=128), a 131072-token chunked prefill in chunks of
+512 with l_I=128, l_L=2048, k=4096, eps=3, mixture keys with planted needle
+spans.  One bench "step" is the whole chunked prefill of one layer: 256 ESA steps,
+each = esa_compress_keys + esa_select + esa_attend.  The metric is prefill
+tokens/s through the 32-layer stack (= 131072 / (32 x layer time)); the layers
+are independent and identically shaped, and the timed steps cycle over
+``--layers`` distinct layers' data.  The decode workload ("c3": 8 sequences x
+131072 cached tokens, one query each, 256 steps) is timed in the same run and
+reported under "decode".
+
+Launch: ``python bench.py --gpus N --steps K --warmup W``; for N > 1 under
+torchrun, one rank per GPU, every rank an independent replica of the workload
+(the step has no cross-GPU exchange), value = total tokens / max-over-ranks time.
+``--impl reference`` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import esa_synth as syn
+
+N_LAYERS_STACK = 32
+
+
+# ----------------------------------------------------------------------------
+# small helpers (also exercised by the CPU tests)
+# ----------------------------------------------------------------------------
+def shard_units(total: int, rank: int, world: int):
+    """Contiguous share [lo, hi) of ``total`` independent units for ``rank``."""
+    base, rem = divmod(total, world)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "tflops_burst": p["bf16_tflops"],
+                "tflops_sustained": p["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def attend_flops(cfg, t: int, l_C: int) -> float:
+    """Algorithmic flops of one esa_attend launch: 4 d_H l_C (n_att - l_C/2)."""
+    i_end = min(cfg.l_I, t)
+    m_end = max(i_end, t - cfg.l_L)
+    n_att = i_end + min(cfg.k, m_end - i_end) + (t - m_end) + l_C
+    return 4.0 * cfg.d_H * l_C * (n_att - l_C / 2.0)
+
+
+def score_flops(cfg, t: int, l_C: int) -> float:
+    """One scoring pass (the method's own count): 2 l_C l_M d' + l_C l_M."""
+    i_end = min(cfg.l_I, t)
+    l_M = max(i_end, t - cfg.l_L) - i_end
+    return (2.0 * cfg.d_c + 1.0) * l_C * l_M if l_M > cfg.k else 0.0
+
+
+def decode_bytes(cfg, t: int) -> float:
+    """Algorithmic HBM bytes of one decode step of one sequence: 2 l_M d' + 4 n_att d_G."""
+    i_end = min(cfg.l_I, t)
+    m_end = max(i_end, t - cfg.l_L)
+    l_M = m_end - i_end
+    n_att = i_end + min(cfg.k, l_M) + (t - m_end) + 1
+    return 2.0 * l_M * cfg.d_c + 4.0 * n_att * cfg.d_G
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------
+# workloads on the device
+# ----------------------------------------------------------------------------
+def bits_to_dev(bits, pin=False):
+    t = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+    return t.pin_memory() if pin else t.cuda()
+
+
+class PrefillLayer:
+    """One layer of a prefill workload: Q/K/V resident in HBM, caches sized for S tokens."""
+
+    def __init__(self, cfg, layer, keep_host=False):
+        S = cfg.S
+        self.cfg = cfg
+        qb = syn.qkv_rows(cfg, "q", 0, S, layer)
+        kb = syn.qkv_rows(cfg, "k", 0, S, layer)
+        vb = syn.qkv_rows(cfg, "v", 0, S, layer)
+        self.Q = bits_to_dev(qb)[None]          # [1,S,H,d]
+        self.K = bits_to_dev(kb)[None]          # [1,S,H_G,d]  (the K cache; C's rows are in place)
+        self.V = bits_to_dev(vb)[None]
+        self.host = None
+        if keep_host:
+            self.host = tuple(bits_to_dev(x, pin=True) for x in (qb, kb, vb))
+        self.wq, self.wk = syn.compressor_weights(cfg, layer)
+
+
+def make_ctx(cfg, max_tokens, max_chunk, max_batch):
+    import paper_2502_14477_b200 as esa
+    return esa.Esa(esa.EsaConfig(cfg.H, cfg.H_G, cfg.d, cfg.d_c, cfg.l_I, cfg.l_L, cfg.k, cfg.eps,
+                                 max_chunk, max_batch, max_tokens))
+
+
+def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
+    """The whole chunked prefill of one layer with inputs resident in HBM."""
+    Kc, idx, n_sel, O = bufs
+    for t in range(0, cfg.S, cfg.l_C):
+        l_C = min(cfg.l_C, cfg.S - t)
+        Qc = L.Q[:, t: t + l_C]
+        ctx.compress_keys(L.K[:, t: t + l_C], Kc, [t])
+        ctx.select(Qc, Kc, [t], idx, n_sel)
+        if attend_events is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        ctx.attend(Qc, L.K, L.V, [t], idx, n_sel, O[:, t: t + l_C])
+        if attend_events is not None:
+            e1.record()
+            attend_events.append((t, l_C, e0, e1))
+
+
+def run_prefill_layer_e2e(ctx, cfg, L, bufs, caches, stage, O_host):
+    """Same work with HOST inputs and outputs: every chunk's Q/K/V rows are copied from
+    pinned host memory, appended to the device caches, and the chunk's output is copied back."""
+    Kc, idx, n_sel, _ = bufs
+    Kcache, Vcache = caches
+    Qs, Ks, Vs, Os = stage
+    hq, hk, hv = L.host
+    for t in range(0, cfg.S, cfg.l_C):
+        l_C = min(cfg.l_C, cfg.S - t)
+        Qs[0, :l_C].copy_(hq[t: t + l_C], non_blocking=True)
+        Ks[0, :l_C].copy_(hk[t: t + l_C], non_blocking=True)
+        Vs[0, :l_C].copy_(hv[t: t + l_C], non_blocking=True)
+        ctx.append_kv(Ks[:, :l_C], Vs[:, :l_C], Kcache, Vcache, [t])
+        ctx.compress_keys(Ks[:, :l_C], Kc, [t])
+        ctx.select(Qs[:, :l_C], Kc, [t], idx, n_sel)
+        ctx.attend(Qs[:, :l_C], Kcache, Vcache, [t], idx, n_sel, Os[:, :l_C])
+        O_host[t: t + l_C].copy_(Os[0, :l_C], non_blocking=True)
+
+
+# ----------------------------------------------------------------------------
+# the two arms
+# ----------------------------------------------------------------------------
+def oracle_sample(cfg, layer, chunks, heads=None):
+    """Times the CPU oracle on a few chunks of the prefill workload; returns
+    (tokens processed, seconds, description)."""
+    from oracle import esa_oracle as orc
+    wq, wk = syn.compressor_weights(cfg, layer)
+    Wq, Wk = orc.bf16_round(wq), orc.bf16_round(wk)
+    p = orc.EsaParams(cfg.l_I, cfg.l_L, cfg.k, cfg.eps)
+    t_max = max(chunks) * cfg.l_C + cfg.l_C
+    K = syn.bf16_bits_to_f64(syn.qkv_rows(cfg, "k", 0, t_max, layer))
+    V = syn.bf16_bits_to_f64(syn.qkv_rows(cfg, "v", 0, t_max, layer))
+    Kc = orc.compress(K.reshape(t_max, -1), Wk)          # the cache carried between steps
+    secs, toks = 0.0, 0
+    for c in chunks:
+        t = c * cfg.l_C
+        Q = syn.bf16_bits_to_f64(syn.qkv_rows(cfg, "q", t, t + cfg.l_C, layer))
+        t0 = time.perf_counter()
+        orc.esa_step(Q, K[: t + cfg.l_C], V[: t + cfg.l_C], Wq, Wk, p, t, Kc=Kc, heads=heads)
+        secs += time.perf_counter() - t0
+        toks += cfg.l_C
+    return toks, secs, f"chunks {list(chunks)} of layer {layer} (all heads), k' cache precomputed"
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    chunks = [13, 255]                       # first chunk with l_M > k, and the last
+    total = args.steps + args.warmup
+    secs_all = []
+    for s in range(total):
+        toks, secs, what = oracle_sample(cfg, s % 2, chunks)
+        if s >= args.warmup:
+            secs_all.append(secs / toks)
+    per_tok = sum(secs_all) / len(secs_all)
+    value = 1.0 / (per_tok * N_LAYERS_STACK)
+    line = {
+        "impl": "reference", "metric": "esa_prefill_tokens_per_s_128k", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * per_tok * len(chunks) * cfg.l_C, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"each step: {what}; per-token time extrapolated to the 32-layer stack"},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(cfg):
+    return {"workload": "c5: Llama-3-8B attention shape, 131072-token prefill in chunks of 512, "
+                        "l_I=128 l_L=2048 k=4096 eps=3 d'=128, mixture keys + planted needles; "
+                        "a step = one layer's whole chunked prefill, value = tokens/s through 32 such layers",
+            "H": cfg.H, "H_G": cfg.H_G, "head_dim": cfg.d, "d_c": cfg.d_c, "l_C": cfg.l_C, "S": cfg.S,
+            "l2": "per-layer inputs (1.6 GB) exceed the 126 MB L2; steps cycle over distinct layers"}
+
+
+def time_decode(cfg3, n_steps, rank_seed):
+    """Config c3: B sequences with S cached tokens, n_steps decode steps (append K/V,
+    compress the new key, select, attend).  Returns (us/step, bytes/step, launches/step)."""
+    B, S = cfg3.B, cfg3.S
+    n = S + n_steps
+    ctx = make_ctx(cfg3, n, 1, B)
+    wq, wk = syn.compressor_weights(cfg3)
+    ctx.set_compressors(wq, None, wk, None)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(cfg3.seed + 1000 * rank_seed)
+    # decode inputs are N(0,1) bf16; drawn on the device (2 x 2.2 GB) to keep start-up short
+    K = torch.randn(B, n, cfg3.H_G, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
+    V = torch.randn(B, n, cfg3.H_G, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
+    Qs = torch.randn(n_steps, B, 1, cfg3.H, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
+    Knew = K[:, S:].clone()
+    Vnew = V[:, S:].clone()
+    Kc = torch.zeros(B, n, cfg3.d_c, dtype=torch.bfloat16, device="cuda")
+    for r0 in range(0, S, 4096):
+        ctx.compress_keys(K[:, r0: r0 + 4096].contiguous(), Kc, [r0] * B)
+    idx = torch.zeros(B, cfg3.k, dtype=torch.int32, device="cuda")
+    n_sel = torch.zeros(B, dtype=torch.int32, device="cuda")
+    O = torch.empty(B, 1, cfg3.H, cfg3.d, dtype=torch.bfloat16, device="cuda")
+
+    def step(i):
+        t = [S + i] * B
+        kn, vn = Knew[:, i: i + 1], Vnew[:, i: i + 1]
+        ctx.append_kv(kn.contiguous(), vn.contiguous(), K, V, t)
+        ctx.compress_keys(kn.contiguous(), Kc, t)
+        ctx.select(Qs[i], Kc, t, idx, n_sel)
+        ctx.attend(Qs[i], K, V, t, idx, n_sel, O)
+
+    for i in range(min(8, n_steps)):
+        step(i)
+    torch.cuda.synchronize()
+    l0 = ctx.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n_steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / n_steps
+    byts = B * sum(decode_bytes(cfg3, S + i) for i in range(n_steps)) / n_steps
+    launches = (ctx.launch_count - l0) / n_steps
+    assert ctx.last_device_status() == 0
+    ctx.close()
+    return us, byts, launches
+
+
+def run_esa(args, cfg):
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+
+    n_res = max(1, min(args.layers, args.steps + args.warmup))
+    layers = [PrefillLayer(cfg, (rank * n_res + i) % N_LAYERS_STACK, keep_host=(i == 0)) for i in range(n_res)]
+    ctx = make_ctx(cfg, cfg.S, cfg.l_C, 1)
+    Kc = torch.zeros(1, cfg.S, cfg.d_c, dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros(1, cfg.k, dtype=torch.int32, device="cuda")
+    n_sel = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O = torch.empty(1, cfg.S, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda")
+    bufs = (Kc, idx, n_sel, O)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step(i, ev=None):
+        L = layers[i % n_res]
+        ctx.set_compressors(L.wq, None, L.wk, None)
+        run_prefill_layer(ctx, cfg, L, bufs, ev)
+
+    for i in range(args.warmup):
+        one_step(i)
+    sync_all()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count
+    events = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for i in range(args.steps):
+        one_step(args.warmup + i, events)
+    e1.record()
+    sync_all()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), "cuda" if world > 1 else None)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = ctx.launch_count - launches0
+    assert ctx.last_device_status() == 0
+    ms_per_step = ms_total / args.steps
+    value = world * cfg.S / (N_LAYERS_STACK * ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (the attention launches), timed inside the region above
+    att_ms = sum(a.elapsed_time(b) for (_, _, a, b) in events)
+    att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
+    achieved = att_flops / (att_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attend_kernel", "achieved": achieved, "peak": peaks["tflops_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": None,
+                "peak_source": peaks["source"] + " sustained bf16", "share_of_step": att_ms / (ms_total),
+                "launches": len(events)}
+
+    # end to end: host inputs and outputs
+    L0 = layers[0]
+    caches = (torch.zeros_like(L0.K), torch.zeros_like(L0.V))
+    stage = (torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"),
+             torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
+             torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
+             torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"))
+    O_host = torch.empty(cfg.S, cfg.H, cfg.d, dtype=torch.bfloat16).pin_memory()
+    ctx.set_compressors(L0.wq, None, L0.wk, None)
+    run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host)
+    sync_all()
+    n_e2e = max(1, min(2, args.steps))
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(n_e2e):
+        run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host)
+    t1.record()
+    sync_all()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1), "cuda" if world > 1 else None) / n_e2e
+    h2d = cfg.S * (cfg.d_H + 2 * cfg.d_G) * 2
+    d2h = cfg.S * cfg.d_H * 2
+    e2e = {"value": world * cfg.S / (N_LAYERS_STACK * e2e_ms * 1e-3), "unit": "tokens/s",
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
+    del caches, stage, layers
+    ctx.close()
+    torch.cuda.empty_cache()
+
+    # decode workload (config c3)
+    decode = None
+    if not args.no_decode:
+        cfg3 = syn.get_config("c3")
+        us, byts, lps = time_decode(cfg3, args.decode_steps, rank)
+        us = max_over_ranks(us, "cuda" if world > 1 else None)
+        gbs = byts / (us * 1e-6) / 1e9
+        decode = {"workload": "c3: 8 sequences x 131072 cached tokens, 1 query each, k=4096 l_L=2048 l_I=128",
+                  "us_per_step": us, "steps": args.decode_steps, "launches_per_step": lps,
+                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                               "algorithmic_bytes_per_step": byts, "peak_source": peaks["source"] + " copy"}}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    # CPU oracle on a bounded sample of the same workload
+    toks, secs, what = oracle_sample(cfg, 0, [13, 255])
+    cpu = {"value": toks / secs / N_LAYERS_STACK, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+           "sample": what + "; per-token time extrapolated to the 32-layer stack"}
+    line = {
+        "metric": "esa_prefill_tokens_per_s_128k", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "cpu_baseline": cpu, "decode": decode,
+        "per_layer_tokens_per_s": world * cfg.S / (ms_per_step * 1e-3),
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="esa", choices=["esa", "reference"])
+    ap.add_argument("--layers", type=int, default=3, help="distinct layers' data kept resident")
+    ap.add_argument("--decode-steps", type=int, default=256)
+    ap.add_argument("--no-decode", action="store_true")
+    args = ap.parse_args()
+    cfg = syn.get_config("c5")
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the ESA path has no CPU fallback "
+                             "(use --impl reference for the CPU oracle)")
+        run_esa(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -7,9 +7,10 @@ Comparison rules
     max_c |r_c|): the aggregated score is a difference of numbers of size |r_c| and the
     k-th score is often exactly 0, so the relative band is taken against the larger.
   * attention outputs: max-abs <= 2e-2 and mean-abs <= 2e-3 (bf16 output).
-  * compressed keys: bit-exact bf16, except elements whose exact (float64) value lies
-    within ``delta`` of a bf16 rounding boundary, where the neighbouring bf16 value is
-    accepted (the kernel accumulates in fp32, the oracle in float64).
+  * compressed keys: bit-exact bf16, except that the kernel's value may be the bf16
+    rounding of any number within the fp32 accumulation bound of the exact (float64)
+    product (the kernel accumulates in fp32, the oracle in float64); at most 0.2 % of
+    the elements may differ at all.
 """
 from __future__ import annotations
 
@@ -98,14 +99,18 @@ def check_compressed(kc_gpu: torch.Tensor, X: np.ndarray, W: np.ndarray, b=None,
     neq = got != want
     if not neq.any():
         return 0
-    # fp32 accumulation error bound: d_in terms, each product exact, sum error <= d_in * 2^-24 * sum|terms|
+    # The kernel accumulates in fp32: its sum lies within d_in * 2^-24 * sum|terms| of the exact
+    # one, so its bf16 result must be the rounding of SOME value in that interval (rounding is
+    # monotone, so it suffices to round the interval's ends).
     bound = X.shape[1] * 2.0 ** -24 * (np.abs(X) @ np.abs(W).T)
-    ulp = np.abs(np.spacing(want.astype(np.float32)).astype(np.float64)) * 2.0 ** 16   # bf16 ulp at `want`
-    # distance of the exact value from the rounding boundary on the side of `got`
-    boundary = (want + got) / 2.0
-    ok = (np.abs(got - want) <= 1.0001 * ulp) & (np.abs(exact - boundary) <= bound + 1e-30)
-    bad = neq & ~ok
-    assert not bad.any(), f"{what}: {int(bad.sum())} compressed values differ beyond the rounding-boundary rule"
+    if b is not None:
+        bound = bound + 2.0 ** -24 * np.abs(exact)
+    lo, hi = orc.bf16_round(exact - bound), orc.bf16_round(exact + bound)
+    bad = (got < lo) | (got > hi)
+    assert not bad.any(), (f"{what}: {int(bad.sum())} of {int(neq.sum())} differing compressed values are not a "
+                           f"bf16 rounding of a value within the fp32 accumulation bound; (exact, want, got) = "
+                           f"{list(zip(exact[bad][:4], want[bad][:4], got[bad][:4]))}")
+    assert neq.mean() < 2e-3, f"{what}: {neq.mean():.2e} of the compressed values differ from the exact rounding"
     return int(neq.sum())
 
 
