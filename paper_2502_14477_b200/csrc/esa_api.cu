@@ -29,14 +29,13 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, part, rkey, skey, pkey, att, status, total;
-    size_t part_elems, att_elems;
+    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, att, status, total;
+    size_t att_elems;
 };
 
 Layout make_layout(const esa_config* c) {
     Layout L;
     const size_t dH = (size_t)c->n_q_heads * c->head_dim, dG = (size_t)c->n_kv_heads * c->head_dim;
-    const size_t rows_max = (size_t)c->max_batch * (c->max_chunk > kCompressMaxRows ? c->max_chunk : kCompressMaxRows);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
     L.wq = take(2 * c->d_c * dH);
@@ -44,11 +43,6 @@ Layout make_layout(const esa_config* c) {
     L.bq = take(4 * c->d_c);
     L.bk = take(4 * c->d_c);
     L.qc = take(2 * (size_t)c->max_batch * c->max_chunk * c->d_c);
-    // split-K partials: up to 16 splits of the largest compression
-    L.part_elems = (size_t)16 * rows_max * c->d_c;
-    if (L.part_elems > (size_t)64 << 20) L.part_elems = (size_t)64 << 20;   // 256 MB cap
-    if (L.part_elems < rows_max * c->d_c) L.part_elems = rows_max * c->d_c;
-    L.part = take(4 * L.part_elems);
     L.rkey = take(4 * (size_t)c->max_batch * c->max_chunk);
     L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
@@ -156,8 +150,6 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->bq = reinterpret_cast<float*>(base + L.bq);
     c->bk = reinterpret_cast<float*>(base + L.bk);
     c->Qc = reinterpret_cast<__nv_bfloat16*>(base + L.qc);
-    c->part = reinterpret_cast<float*>(base + L.part);
-    c->part_elems = L.part_elems;
     c->rkey = reinterpret_cast<uint32_t*>(base + L.rkey);
     c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);

@@ -291,20 +291,24 @@ static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     constexpr int BM = NW * 16;
     const int R = p.l_C * p.G;
     const int row_tiles = (R + BM - 1) / BM;
+    constexpr int smem = (BM + 4 * BN) * (D / 8) * 16;
+    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
     int nsplit = 1;
     if (R <= kAttSplitRows && row_tiles == 1) {
+        // split the key list so that one wave of CTAs fills the machine (never a second, short wave)
+        int per_sm = 1;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN>, NW * 32, smem);
+        if (e != cudaSuccess) return e;
         const int ctas = p.HG * B;
         const int n_tiles = (n_att_max + BN - 1) / BN;
-        nsplit = (6 * ctx->num_sms + ctas - 1) / ctas;
+        nsplit = (per_sm * ctx->num_sms) / ctas;
         if (nsplit > kAttMaxSplits) nsplit = kAttMaxSplits;
         if (nsplit > n_tiles) nsplit = n_tiles;
         while (nsplit > 1 && (size_t)B * p.HG * nsplit * R * (D + 2) > ctx->att_part_elems) --nsplit;
         if (nsplit < 1) nsplit = 1;
     }
     p.nsplit = nsplit;
-    constexpr int smem = (BM + 4 * BN) * (D / 8) * 16;
-    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
     attend_kernel<D, NW, BN><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
     ctx->launches += 1;
     if (nsplit > 1) {

@@ -6,9 +6,14 @@
 // X is [rows, d_in] (heads concatenated, Section 3.1 "Efficient Selection"), W is
 // [d_c, d_in]; both are K-major, so the product is a TN GEMM.  The output is only d_c
 // wide, so a chunk yields very few output tiles; the reduction dimension is therefore
-// split across CTAs, each writing an fp32 partial tile, and a second kernel adds the
-// partials in a fixed order (deterministic), adds the bias and rounds to bf16.
+// split across the CTAs of a thread-block cluster; each keeps its fp32 partial tile in
+// shared memory and the cluster adds the partials through distributed shared memory in a
+// fixed order (deterministic), adds the bias and rounds to bf16.  No global scratch.
+#include <cooperative_groups.h>
+
 #include "esa_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace esa {
 
@@ -18,8 +23,9 @@ constexpr int CP_THREADS = 128;
 
 template <int DC>
 __global__ void __launch_bounds__(CP_THREADS)
-compress_partial_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
-                        float* __restrict__ part, int rows, int d_in, int kslice) {
+compress_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
+                const float* __restrict__ bias, __nv_bfloat16* __restrict__ dst, int rows, int rows_per_seq,
+                int d_in, int kslice, int64_t seq_stride, RowMap map) {
     constexpr int CH = CP_BK / 8;  // 16-byte chunks per smem row
     extern __shared__ uint4 smem[];
     uint4* sX[2] = {smem, smem + CP_BM * CH};
@@ -79,39 +85,42 @@ compress_partial_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16
         __syncthreads();
     }
 
-    // fp32 partial tile -> part[split][row][DC]
-    const int r_lo = row0 + warp * 16 + (lane >> 2);
-    float* base = part + (size_t)split * rows * DC;
+    // fp32 partial tile -> this CTA's shared memory
+    float* sPart = reinterpret_cast<float*>(smem + 2 * (CP_BM + DC) * CH);   // [CP_BM][DC]
+    {
+        const int r = warp * 16 + (lane >> 2);
 #pragma unroll
-    for (int nb = 0; nb < DC / 8; ++nb) {
-        int col = nb * 8 + (lane & 3) * 2;
-        if (r_lo < rows) *reinterpret_cast<float2*>(base + (size_t)r_lo * DC + col) = make_float2(acc[nb][0], acc[nb][1]);
-        if (r_lo + 8 < rows)
-            *reinterpret_cast<float2*>(base + (size_t)(r_lo + 8) * DC + col) = make_float2(acc[nb][2], acc[nb][3]);
+        for (int nb = 0; nb < DC / 8; ++nb) {
+            int col = nb * 8 + (lane & 3) * 2;
+            *reinterpret_cast<float2*>(sPart + r * DC + col) = make_float2(acc[nb][0], acc[nb][1]);
+            *reinterpret_cast<float2*>(sPart + (r + 8) * DC + col) = make_float2(acc[nb][2], acc[nb][3]);
+        }
     }
-}
-
-// Adds the split-K partials in split order, adds the bias, rounds to bf16 and writes row
-// i of sequence b to dst row b * seq_stride + row0[b] + i.
-__global__ void compress_finalize_kernel(const float* __restrict__ part, const float* __restrict__ bias,
-                                         __nv_bfloat16* __restrict__ dst, int rows, int rows_per_seq,
-                                         int dc, int nsplit, int64_t seq_stride, RowMap map) {
-    const int per_row = dc / 4;
-    int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (gid >= (int64_t)rows * per_row) return;
-    int row = (int)(gid / per_row), c4 = (int)(gid % per_row) * 4;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int sp = 0; sp < nsplit; ++sp) {
-        float4 v = *reinterpret_cast<const float4*>(part + ((size_t)sp * rows + row) * dc + c4);
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    // The CTAs of a cluster hold the split-K partials of one row tile.  Each CTA sums a
+    // band of rows over all of them through distributed shared memory, in split order (so
+    // the result does not depend on timing), adds the bias and rounds to bf16.
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();
+    const int nsplit = gridDim.y;
+    const int band = CP_BM / nsplit;                  // rows reduced by this CTA
+    constexpr int PER_ROW = DC / 4;
+    for (int i = tid; i < band * PER_ROW; i += CP_THREADS) {
+        const int lr = split * band + i / PER_ROW, c4 = (i % PER_ROW) * 4;
+        const int row = row0 + lr;
+        if (row >= rows) continue;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp = 0; sp < nsplit; ++sp) {
+            const float4 v = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sPart, sp) + lr * DC + c4);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        if (bias) {
+            s.x += bias[c4]; s.y += bias[c4 + 1]; s.z += bias[c4 + 2]; s.w += bias[c4 + 3];
+        }
+        const int b = row / rows_per_seq, ii = row % rows_per_seq;
+        __nv_bfloat16* o = dst + ((int64_t)b * seq_stride + map.row0[b] + ii) * DC + c4;
+        *reinterpret_cast<uint2*>(o) = make_uint2(pack_bf16(s.x, s.y), pack_bf16(s.z, s.w));
     }
-    if (bias) {
-        s.x += bias[c4]; s.y += bias[c4 + 1]; s.z += bias[c4 + 2]; s.w += bias[c4 + 3];
-    }
-    int b = row / rows_per_seq, i = row % rows_per_seq;
-    __nv_bfloat16* o = dst + ((int64_t)b * seq_stride + map.row0[b] + i) * dc + c4;
-    uint2 pk = make_uint2(pack_bf16(s.x, s.y), pack_bf16(s.z, s.w));
-    *reinterpret_cast<uint2*>(o) = pk;
+    cluster.sync();    // shared memory stays alive until every remote read is done
 }
 
 template <int DC>
@@ -121,29 +130,29 @@ static cudaError_t launch_compress_t(esa_ctx* ctx, const __nv_bfloat16* X, int r
                                      cudaStream_t st) {
     const int row_tiles = (rows + CP_BM - 1) / CP_BM;
     const int nk_total = d_in / CP_BK;
-    // split the reduction so that about two CTAs per SM are in flight
+    // split the reduction over a cluster of up to 8 CTAs while that still adds CTAs usefully
     int nsplit = 1;
-    while (nsplit * 2 <= nk_total && (nk_total % (nsplit * 2)) == 0 &&
-           row_tiles * nsplit * 2 <= 2 * ctx->num_sms &&
-           (size_t)(nsplit * 2) * rows * DC <= ctx->part_elems)
-        nsplit *= 2;
-    if ((size_t)nsplit * rows * DC > ctx->part_elems) return cudaErrorInvalidValue;
+    while (nsplit < 8 && (nk_total % (nsplit * 2)) == 0 && row_tiles * nsplit < 2 * ctx->num_sms) nsplit *= 2;
     const int kslice = d_in / nsplit;
-    constexpr int smem = 2 * (CP_BM + DC) * (CP_BK / 8) * 16;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(compress_partial_kernel<DC>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    compress_partial_kernel<DC><<<dim3(row_tiles, nsplit), CP_THREADS, smem, st>>>(X, W, ctx->part, rows,
-                                                                                  d_in, kslice);
-    const int64_t n = (int64_t)rows * (DC / 4);
-    compress_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
-        ctx->part, bias, dst, rows, rows_per_seq, DC, nsplit, seq_stride, map);
-    ctx->launches += 2;
-    return cudaGetLastError();
+    constexpr int smem = 2 * (CP_BM + DC) * (CP_BK / 8) * 16 + CP_BM * DC * 4;
+    cudaError_t e = cudaFuncSetAttribute(compress_kernel<DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(row_tiles, nsplit);
+    cfg.blockDim = dim3(CP_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = nsplit;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, compress_kernel<DC>, X, W, bias, dst, rows, rows_per_seq, d_in, kslice,
+                           seq_stride, map);
+    ctx->launches += 1;
+    return e;
 }
 
 cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,

@@ -35,8 +35,6 @@ struct esa_ctx {
     float* bq;           // [dc]
     float* bk;           // [dc]
     __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
-    float* part;         // split-K partial sums of the compression GEMM
-    size_t part_elems;
     uint32_t* rkey;      // [max_batch * max_chunk] ordered keys of the row maxima r_c
     uint32_t* skey;      // [max_batch, max_tokens] aggregated scores (ordered keys), or raw fp32 S (l_C = 1)
     uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys

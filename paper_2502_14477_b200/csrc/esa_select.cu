@@ -7,8 +7,8 @@
 // pooling copies every peak to 2*eps+1 neighbours), so the order is total: larger score
 // first, lower index first among equal scores.  Scores are handled as order-preserving
 // uint32 keys.  One thread-block cluster works on one sequence: every CTA pools its
-// slice of M, then three radix passes (11 + 11 + 10 bits, histograms combined through
-// distributed shared memory) find the k-th largest key T, and an index-ordered
+// slice of M, then three radix passes (11 + 11 + 10 bits, each digit's histogram all-reduced
+// into every CTA through distributed shared memory) find the k-th largest key T, and an index-ordered
 // compaction emits every key > T plus the first (k - #greater) keys == T, which is
 // exactly "lowest index wins" and leaves the output ascending.
 #include <cooperative_groups.h>
@@ -34,6 +34,7 @@ struct SelectParams {
     int eps;
     int raw;
     int l_C;
+    int slice_cap;          // keys of a CTA's slice that fit in its dynamic shared memory (0: none)
     SeqMeta meta;
 };
 
@@ -43,6 +44,65 @@ __device__ __forceinline__ uint32_t load_agg_key(const uint32_t* src, int m, int
     return v;
 }
 
+// Histogram update aggregated over the warp: pooled scores crowd into a handful of bins
+// (same sign and exponent), so lanes with equal bins elect one leader that adds their count.
+// Must be called by converged lanes named in `active`.
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t bin, uint32_t active) {
+    const uint32_t peers = __match_any_sync(active, bin);
+    if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+}
+
+// Finds, in the cluster-wide histogram `g` of one digit (nb bins, larger bin = larger key),
+// the bin holding the krem-th largest remaining key.  Every CTA runs this on its own copy
+// and gets the same answer.  Returns through sh_out[0] (bin) and sh_out[1] (keys still to
+// place inside that bin).
+__device__ __forceinline__ void find_bin(const uint32_t* g, int nb, uint32_t krem, uint32_t* scan_tmp,
+                                         uint32_t* sh_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // each thread owns `per` consecutive bins, highest bins first
+    const int per = (nb + SEL_THREADS - 1) / SEL_THREADS;
+    uint32_t mine = 0;
+    for (int j = 0; j < per; ++j) {
+        int bin = nb - 1 - (tid * per + j);
+        if (bin >= 0) mine += g[bin];
+    }
+    uint32_t incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+    }
+    if (lane == 31) scan_tmp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = scan_tmp[lane];
+        uint32_t wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += n;
+        }
+        scan_tmp[lane] = wi - w;   // exclusive warp offsets
+    }
+    __syncthreads();
+    const uint32_t before = scan_tmp[warp] + incl - mine;   // keys in bins above this thread's bins
+    if (before < krem && before + mine >= krem) {
+        uint32_t acc = before;
+        for (int j = 0; j < per; ++j) {
+            int bin = nb - 1 - (tid * per + j);
+            if (bin < 0) break;
+            uint32_t c = g[bin];
+            if (acc + c >= krem) {
+                sh_out[0] = (uint32_t)bin;
+                sh_out[1] = krem - acc;
+                break;
+            }
+            acc += c;
+        }
+    }
+    __syncthreads();
+}
+
 __global__ void __cluster_dims__(SEL_CLUSTER, 1, 1) __launch_bounds__(SEL_THREADS)
 select_topk_kernel(SelectParams p) {
     cg::cluster_group cluster = cg::this_cluster();
@@ -50,10 +110,12 @@ select_topk_kernel(SelectParams p) {
     const int b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    __shared__ uint32_t hist[SEL_BINS];
+    extern __shared__ uint32_t slice_keys[];   // pooled keys of this CTA's slice (when they fit)
+    __shared__ uint32_t hist[SEL_BINS];        // this CTA's histogram of the current digit
+    __shared__ uint32_t ghist[3][SEL_BINS];    // cluster-wide histograms, one per digit, same in every CTA
     __shared__ uint32_t warp_cnt[2][32];
-    __shared__ uint32_t cta_cnt[2];          // (#greater, #equal) in this CTA's slice
-    __shared__ uint32_t sh_prefix, sh_krem;  // valid in rank 0: key prefix found so far, k still to place
+    __shared__ uint32_t cta_cnt[2];            // (#greater, #equal) in this CTA's slice
+    __shared__ uint32_t sh_found[2];
     __shared__ uint32_t scan_tmp[SEL_THREADS / 32];
 
     const int i_end = p.meta.i_end[b];
@@ -74,95 +136,81 @@ select_topk_kernel(SelectParams p) {
     const int lo = min(l_M, rank * rows_per_cta * 32);
     const int hi = min(l_M, (rank + 1) * rows_per_cta * 32);
 
-    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) {
+        hist[i] = 0;
+        ghist[0][i] = ghist[1][i] = ghist[2][i] = 0;
+    }
+    cluster.sync();     // every CTA's histograms are zero before anyone adds to them remotely
 
-    // ---- pass 0: pool (Eq. 8), store pooled keys, histogram of bits 31..21
-    for (int m = lo + tid; m < hi; m += SEL_THREADS) {
-        uint32_t best = load_agg_key(src, m, raw, r0);
-        for (int o = 1; o <= p.eps; ++o) {
-            if (m - o >= 0) best = max(best, load_agg_key(src, m - o, raw, r0));
-            if (m + o < l_M) best = max(best, load_agg_key(src, m + o, raw, r0));
+    // ---- digit 0: pool (Eq. 8), store pooled keys, histogram of bits 31..21
+    // A warp loads 32 consecutive keys starting eps before its first output and slides the
+    // window with shuffles: lane i ends with max(key[i .. i+2*eps]) = s' of token first+i, so
+    // each key is loaded and converted once; 32 - 2*eps outputs per step.  Positions outside
+    // M contribute key 0, which is below every real key (the window is clipped to M).
+    // Later passes re-read the slice: from shared memory when it fits, else from pkey (L2).
+    const bool in_smem = (hi - lo) <= p.slice_cap;
+    const uint32_t* keys = in_smem ? slice_keys : pk + lo;     // keys[i] = s' of token lo + i
+    {
+        const int eps = p.eps;
+        const int outs = 32 - 2 * eps;
+        constexpr int UN = 4;                                   // independent loads in flight per lane
+        const int step = (SEL_THREADS / 32) * outs;
+        for (int first0 = lo + warp * outs; first0 < hi; first0 += UN * step) {
+            uint32_t key[UN];
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int mload = first0 + u * step - eps + lane;
+                key[u] = (first0 + u * step < hi && mload >= 0 && mload < l_M) ? load_agg_key(src, mload, raw, r0) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int first = first0 + u * step;
+                if (first >= hi) break;                         // uniform over the warp
+                uint32_t best = key[u];
+                for (int o = 1; o <= 2 * eps; ++o) best = max(best, __shfl_down_sync(0xffffffffu, key[u], o));
+                const int m = first + lane;
+                const bool valid = lane < outs && m < hi;
+                const uint32_t active = __ballot_sync(0xffffffffu, valid);
+                if (valid) {
+                    pk[m] = best;
+                    if (in_smem) slice_keys[m - lo] = best;
+                    hist_add(hist, best >> 21, active);
+                }
+            }
         }
-        pk[m] = best;
-        atomicAdd(&hist[best >> 21], 1u);
     }
 
     uint32_t prefix = 0, krem = (uint32_t)k;
-    // three digit positions: (shift, bits)
     const int shifts[3] = {21, 10, 0};
     const int nbits[3] = {11, 11, 10};
 #pragma unroll 1
     for (int pass = 0; pass < 3; ++pass) {
-        cluster.sync();   // all histograms of this pass complete
-        if (rank == 0) {
-            // combine the cluster's histograms into rank 0's copy
-            const int nb = 1 << nbits[pass];
-            for (int i = tid; i < nb; i += SEL_THREADS) {
-                uint32_t s = hist[i];
-                for (int r = 1; r < SEL_CLUSTER; ++r) s += *cluster.map_shared_rank(&hist[i], r);
-                hist[i] = s;
+        __syncthreads();
+        // all-reduce of the digit histogram: every non-empty local bin is added to every CTA's copy
+        const int nb = 1 << nbits[pass];
+        for (int i = tid; i < nb; i += SEL_THREADS) {
+            const uint32_t c = hist[i];
+            if (c) {
+                for (int r = 0; r < SEL_CLUSTER; ++r) atomicAdd(cluster.map_shared_rank(&ghist[pass][i], r), c);
             }
-            __syncthreads();
-            // find the bin holding the krem-th largest key: suffix sums from the top bin
-            // each thread owns nb / SEL_THREADS consecutive bins (1 or 2), highest bins first
-            const int per = (nb + SEL_THREADS - 1) / SEL_THREADS;
-            uint32_t mine = 0;
-            for (int j = 0; j < per; ++j) {
-                int bin = nb - 1 - (tid * per + j);
-                if (bin >= 0) mine += hist[bin];
-            }
-            // inclusive scan of "mine" over threads
-            uint32_t incl = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += n;
-            }
-            if (lane == 31) scan_tmp[warp] = incl;
-            __syncthreads();
-            if (warp == 0) {
-                uint32_t w = scan_tmp[lane];
-                uint32_t wi = w;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t n = __shfl_up_sync(0xffffffffu, wi, o);
-                    if (lane >= o) wi += n;
-                }
-                scan_tmp[lane] = wi - w;   // exclusive warp offsets
-            }
-            __syncthreads();
-            uint32_t before = scan_tmp[warp] + incl - mine;   // keys in bins above this thread's bins
-            if (before < krem && before + mine >= krem) {
-                uint32_t acc = before;
-                for (int j = 0; j < per; ++j) {
-                    int bin = nb - 1 - (tid * per + j);
-                    if (bin < 0) break;
-                    uint32_t c = hist[bin];
-                    if (acc + c >= krem) {
-                        sh_prefix = prefix | ((uint32_t)bin << shifts[pass]);
-                        sh_krem = krem - acc;
-                        break;
-                    }
-                    acc += c;
-                }
-            }
-            __syncthreads();
         }
-        cluster.sync();   // rank 0 published (prefix, krem)
-        prefix = *cluster.map_shared_rank(&sh_prefix, 0);
-        krem = *cluster.map_shared_rank(&sh_krem, 0);
-        cluster.sync();   // everyone has read before rank 0's histogram is reused
+        cluster.sync();
+        find_bin(ghist[pass], nb, krem, scan_tmp, sh_found);
+        prefix |= sh_found[0] << shifts[pass];
+        krem = sh_found[1];
         if (pass == 2) break;
-        // ---- next pass: histogram of the next digit among keys matching the prefix
+        // ---- next digit among the keys that match the prefix found so far
         for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
         __syncthreads();
         const int sh = shifts[pass + 1];
         const uint32_t dmask = (1u << nbits[pass + 1]) - 1u;
-        const int psh = shifts[pass];          // bits above psh (inclusive) are fixed
-        for (int m = lo + tid; m < hi; m += SEL_THREADS) {
-            uint32_t key = pk[m];
-            if ((key >> psh) == (prefix >> psh)) atomicAdd(&hist[(key >> sh) & dmask], 1u);
+        const int psh = shifts[pass];          // bits psh and above are fixed
+        for (int m0 = lo + warp * 32; m0 < hi; m0 += SEL_THREADS) {
+            const int m = m0 + lane;
+            const uint32_t key = (m < hi) ? keys[m - lo] : 0u;
+            const bool take = (m < hi) && (key >> psh) == (prefix >> psh);
+            const uint32_t active = __ballot_sync(0xffffffffu, take);
+            if (take) hist_add(hist, (key >> sh) & dmask, active);
         }
     }
     const uint32_t T = prefix;   // k-th largest key; krem of the keys equal to T are taken
@@ -175,7 +223,7 @@ select_topk_kernel(SelectParams p) {
     const int w_hi = min(hi, lo + (warp + 1) * rows_per_warp * 32);
     uint32_t n_gt = 0, n_eq = 0;
     for (int m = w_lo + lane; m < w_hi; m += 32) {
-        uint32_t key = pk[m];
+        uint32_t key = keys[m - lo];
         n_gt += key > T;
         n_eq += key == T;
     }
@@ -211,7 +259,7 @@ select_topk_kernel(SelectParams p) {
     int32_t* out = p.idx_out + (int64_t)b * p.top_k;
     for (int m0 = w_lo; m0 < w_hi; m0 += 32) {
         int m = m0 + lane;
-        uint32_t key = (m < w_hi) ? pk[m] : 0u;
+        uint32_t key = (m < w_hi) ? keys[m - lo] : 0u;
         bool gt = (m < w_hi) && key > T;
         bool eq = (m < w_hi) && key == T;
         uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
@@ -249,13 +297,20 @@ __global__ void read_pooled_kernel(const uint32_t* __restrict__ pkey, float* __r
 
 cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, int32_t* idx_out,
                           int32_t* n_sel_out, cudaStream_t st) {
-    (void)max_lM;
     SelectParams p;
     p.skey = ctx->skey; p.rkey = ctx->rkey; p.pkey = ctx->pkey;
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.top_k = ctx->cfg.top_k; p.eps = ctx->cfg.eps;
     p.raw = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
-    select_topk_kernel<<<dim3(SEL_CLUSTER, B), SEL_THREADS, 0, st>>>(p);
+    // dynamic shared memory for a CTA's slice of pooled keys (largest sequence of the call)
+    const int rows32 = (max_lM + 31) / 32;
+    const int slice = ((rows32 + SEL_CLUSTER - 1) / SEL_CLUSTER) * 32;
+    size_t smem = (size_t)slice * 4;
+    if (smem > 160 * 1024) smem = 0;
+    p.slice_cap = (int)(smem / 4);
+    cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e != cudaSuccess) return e;
+    select_topk_kernel<<<dim3(SEL_CLUSTER, B), SEL_THREADS, smem, st>>>(p);
     ctx->launches += 1;
     return cudaGetLastError();
 }
