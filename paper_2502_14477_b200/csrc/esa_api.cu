@@ -50,6 +50,9 @@ Layout make_layout(const esa_config* c) {
     size_t rows = (size_t)c->max_chunk * G;
     if (rows > (size_t)kAttSplitRows) rows = kAttSplitRows;
     L.att_elems = (size_t)c->max_batch * c->n_kv_heads * kAttMaxSplits * rows * (c->head_dim + 2);
+    // prefill-sized chunks: room for one sequence's key list split kAttPrefillSplits ways
+    const size_t big = (size_t)c->n_kv_heads * kAttPrefillSplits * c->max_chunk * G * (c->head_dim + 2);
+    if ((size_t)c->max_chunk * G > (size_t)kAttSplitRows && big > L.att_elems) L.att_elems = big;
     L.att = take(4 * L.att_elems);
     L.status = take(256);
     L.total = off;

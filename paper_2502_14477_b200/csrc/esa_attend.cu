@@ -334,6 +334,19 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
         if (n > n_att_max) n_att_max = n;
     }
     const int R = l_C * ctx->G;
+    if (R > kAttSplitRows) {
+        // prefill-sized chunks: tcgen05 kernel, then the merge when it split the key list
+        int nsplit = 1;
+        cudaError_t e = launch_attend_tc(ctx, B, l_C, Q, K, V, meta, idx, n_sel, O, n_att_max, st, &nsplit);
+        if (e != cudaSuccess) return e;
+        if (nsplit > 1) {
+            p.nsplit = nsplit;
+            if (ctx->d == 128) attend_merge_kernel<128><<<dim3(R, p.HG, B), 64, 0, st>>>(p);
+            else attend_merge_kernel<64><<<dim3(R, p.HG, B), 32, 0, st>>>(p);
+            ctx->launches += 1;
+        }
+        return cudaGetLastError();
+    }
     if (ctx->d == 128) {
         if (R <= 16) return launch_attend_t<128, 1, 32>(ctx, p, B, n_att_max, st);
         if (R <= 64) return launch_attend_t<128, 4, 64>(ctx, p, B, n_att_max, st);

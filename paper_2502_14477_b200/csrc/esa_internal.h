@@ -12,6 +12,7 @@ namespace esa {
 
 constexpr int kAttMaxSplits = 64;     // split-KV factor of the attention kernel (small chunks)
 constexpr int kAttSplitRows = 64;     // split-KV is used only when l_C * (H/H_G) <= this
+constexpr int kAttPrefillSplits = 4; // largest split of a prefill-sized chunk's key list
 constexpr int kCompressMaxRows = 4096;
 
 // Destination rows of a compression: row i of sequence b goes to
@@ -71,6 +72,13 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
                           const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
                           const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
                           cudaStream_t st);
+
+// Prefill-sized chunks (l_C * H/H_G > kAttSplitRows) on tcgen05; *nsplit_out > 1 means partial
+// results were written to ctx->att_part and the merge kernel must follow.
+cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
+                             const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
+                             const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
+                             int n_att_max, cudaStream_t st, int* nsplit_out);
 
 cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new,
                              const __nv_bfloat16* V_new, int n_new, __nv_bfloat16* K_cache,
