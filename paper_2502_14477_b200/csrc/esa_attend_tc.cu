@@ -4,25 +4,30 @@
 // I u M_k u L u C, C causal), organised for tcgen05:
 //
 //   * A CTA owns 256 rows (row = query c * G + head-in-group g) of one key/value head: two
-//     128-row Q tiles that share every K/V tile brought into shared memory.
-//   * Scores S = Q K^T and outputs O += P V accumulate in tensor memory: per Q tile 128
-//     columns of S and D columns of O (512 columns in all).  P (bf16) overwrites the first
-//     half of its own S columns and is read by the second MMA straight from tensor memory.
+//     128-row Q tiles that share every 64-key K/V tile brought into shared memory.
+//   * Scores S = Q K^T and outputs O += P V accumulate in tensor memory.  Per Q tile: two
+//     64-column S buffers (tile j uses buffer j & 1) and D columns of O, 512 columns in all.
+//     P (bf16) overwrites the first half of its own S buffer and is read by the second MMA
+//     straight from tensor memory.
+//   * Because S is double-buffered, Q K^T of tile j + 2 is issued as soon as P V of tile j
+//     has been issued: the softmax of a Q tile never waits for a product it has just asked
+//     for, and the tensor core works through (Q K^T ahead, P V behind) while both softmax
+//     warpgroups compute.  The kernel is bound by the softmax arithmetic, not by a
+//     softmax -> MMA -> softmax chain.
 //   * Warp roles: warps 0-3 / 4-7 run the online softmax of Q tile 0 / 1 (one thread per
-//     row holding its 128 scores in registers, so row maxima and row sums need no shuffles)
-//     and warps 8-11 gather K/V rows with index-driven 16-byte cp.async into
-//     128-byte-swizzled tiles.  The MMAs of a Q tile are issued by one thread of its own
-//     softmax warpgroup, right after the group has stored P: a separate issuing warp is
-//     starved of issue slots by the arithmetic-heavy softmax warps it shares a scheduler with
-//     (measured: 100-600 cycles per tcgen05.mma instead of 64).  While one Q tile is in its
-//     softmax the tensor core works on the other.
-//   * Half of the exponentials are evaluated on the FMA pipe (Cody-Waite split + cubic), the
-//     rest on the special-function unit, whose 16 results per clock would otherwise bound
-//     the kernel at about half the tensor rate.
+//     row holding its 64 scores in registers, so row maxima and sums need no shuffles),
+//     warps 8-11 gather K/V rows with index-driven 16-byte cp.async into 128-byte-swizzled
+//     tiles, warp 12 issues every MMA.  The issuing warp runs converged (all lanes compute
+//     the warp-uniform descriptors, lane 0 executes the tcgen05 instructions): a single
+//     diverged thread was starved of issue slots by the arithmetic-heavy softmax warps that
+//     share its scheduler (measured 100-600 cycles per tcgen05.mma instead of 64).
+//   * A quarter of the exponentials is evaluated on the FMA pipe (Cody-Waite split + cubic):
+//     measured pipe rates are 8 cycles per warp for ex2 on the special-function unit against
+//     about 10 FMA/ALU-pipe cycles per polynomial element, so the two pipes balance near 1:3.
 //   * The running maximum is only raised when it grows by more than 2^8: until then the
-//     exponentials are taken against the stale maximum (bounded by 256, exact in fp32/bf16
-//     range), which makes rescaling O in tensor memory rare; (O, m, l) stay consistent, so
-//     the final division, or the split merge, needs no correction.
+//     exponentials are taken against the stale maximum (bounded by 256), which makes
+//     rescaling O in tensor memory rare; (O, m, l) stay consistent, so the final division,
+//     or the split merge, needs no correction.
 //   * A long key list can be split across CTAs (blockIdx.z); partial (O, m, l) go to the
 //     context's scratch and the merge kernel of esa_attend.cu combines them.
 #include "esa_internal.h"
@@ -32,22 +37,23 @@ namespace esa {
 
 namespace {
 
-constexpr int TC_BN = 128;            // keys per tile
+constexpr int TC_BN = 64;             // keys per tile
 constexpr int TC_ROWS = 256;          // rows per CTA
+constexpr int TC_STAGES = 4;          // K and V tiles in flight
 constexpr int TC_SOFTMAX_WARPS = 8;
 constexpr int TC_PRODUCER_WARPS = 4;
-constexpr int TC_THREADS = (TC_SOFTMAX_WARPS + TC_PRODUCER_WARPS) * 32;
-// Register split after start-up.  setmaxnreg.inc draws from the pool the CTA was launched with
-// and blocks until the pool can serve it, so the split must fit that pool exactly:
-// launch = 384 threads x 168 registers; 8 warps x 208 + 4 warps x 88 = the same 2016 per lane.
-constexpr int TC_REGS_LAUNCH = 168;
-constexpr int TC_REGS_SOFTMAX = 208;
-constexpr int TC_REGS_OTHER = 88;
-static_assert(TC_SOFTMAX_WARPS * TC_REGS_SOFTMAX + TC_PRODUCER_WARPS * TC_REGS_OTHER <=
-                  (TC_SOFTMAX_WARPS + TC_PRODUCER_WARPS) * TC_REGS_LAUNCH,
-              "register split exceeds the CTA's launch allocation: setmaxnreg.inc would never return");
-constexpr int TC_POLY_PAIRS_OF_4 = 2; // of every 4 column pairs, this many take 2^x on the FMA pipe
+constexpr int TC_MMA_WARP = TC_SOFTMAX_WARPS + TC_PRODUCER_WARPS;
+constexpr int TC_THREADS = 512;       // 13 working warps, padded to whole warpgroups for setmaxnreg
 constexpr int TC_PRODUCERS = TC_PRODUCER_WARPS * 32;
+// Register split after start-up.  setmaxnreg.inc draws from the pool the CTA was launched with
+// and blocks until the pool can serve it, so the split must fit that pool:
+// launch = 16 warps x 128 registers; 8 warps x 168 + 8 warps x 88 = the same 2048 per lane.
+constexpr int TC_REGS_LAUNCH = 128;
+constexpr int TC_REGS_SOFTMAX = 168;
+constexpr int TC_REGS_OTHER = 88;
+static_assert(8 * TC_REGS_SOFTMAX + 8 * TC_REGS_OTHER <= 16 * TC_REGS_LAUNCH,
+              "register split exceeds the CTA's launch allocation: setmaxnreg.inc would never return");
+constexpr int TC_POLY_PAIRS_OF_4 = 1; // of every 4 column pairs, this many take 2^x on the FMA pipe
 constexpr float kRescaleThreshold = 8.0f;    // log2 domain
 
 struct TcAttendParams {
@@ -69,13 +75,16 @@ struct TcAttendParams {
 // barrier slots in shared memory
 enum {
     BAR_Q_FULL = 0,
-    BAR_K_FULL = 1,    // 2
-    BAR_V_FULL = 3,    // 2
-    BAR_K_EMPTY = 5,   // 2
-    BAR_V_EMPTY = 7,   // 2
-    BAR_S_READY = 9,   // 2 (per Q tile)
-    BAR_O_READY = 11,  // 2
-    BAR_COUNT = 13
+    BAR_K_FULL = 1,                         // TC_STAGES
+    BAR_V_FULL = BAR_K_FULL + TC_STAGES,    // TC_STAGES
+    BAR_K_EMPTY = BAR_V_FULL + TC_STAGES,   // TC_STAGES
+    BAR_V_EMPTY = BAR_K_EMPTY + TC_STAGES,  // TC_STAGES
+    BAR_S_READY = BAR_V_EMPTY + TC_STAGES,  // [Q tile][buffer]: 4
+    BAR_P_READY = BAR_S_READY + 4,          // [Q tile][buffer]: 4 (the softmax may run two tiles ahead of
+                                            // the issuing warp, so one barrier per buffer keeps waits adjacent)
+    BAR_PV_DONE = BAR_P_READY + 4,          // per Q tile: 2
+    BAR_O_READY = BAR_PV_DONE + 2,          // per Q tile: 2, completes once
+    BAR_COUNT = BAR_O_READY + 2
 };
 
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
@@ -133,20 +142,23 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
 template <int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attend_tc_kernel(TcAttendParams p) {
-    constexpr int CH = D / 8;                  // 16-byte chunks per row
-    constexpr int TILE_BYTES = TC_BN * D * 2;  // one K or V tile, also one Q tile
-    constexpr int BLK_BYTES = 128 * 128;       // one 64-column block of a 128-row tile
+    constexpr int CH = D / 8;                   // 16-byte chunks per row
+    constexpr int Q_TILE_BYTES = 128 * D * 2;   // one 128-row Q tile
+    constexpr int Q_BLK_BYTES = 128 * 128;      // one 64-column block of it
+    constexpr int KV_TILE_BYTES = TC_BN * D * 2;
+    constexpr int KV_BLK_BYTES = TC_BN * 128;
 
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-    uint8_t* sQ = smem;                           // 2 Q tiles
-    uint8_t* sK = sQ + 2 * TILE_BYTES;            // 2 stages
-    uint8_t* sV = sK + 2 * TILE_BYTES;            // 2 stages
+    uint8_t* sQ = smem;                               // 2 Q tiles
+    uint8_t* sK = sQ + 2 * Q_TILE_BYTES;              // TC_STAGES tiles
+    uint8_t* sV = sK + TC_STAGES * KV_TILE_BYTES;     // TC_STAGES tiles
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int warp_u = __shfl_sync(0xffffffffu, warp, 0);     // provably warp-uniform copy
     const int row0 = blockIdx.x * TC_ROWS;
     const int kvh = blockIdx.y;
     const int b = blockIdx.z / p.nsplit;
@@ -175,13 +187,17 @@ attend_tc_kernel(TcAttendParams p) {
     if (tid == 0) {
         abort_flag = 0;
         mbar_init(bar(BAR_Q_FULL), TC_PRODUCERS);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < TC_STAGES; ++s) {
             mbar_init(bar(BAR_K_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_V_FULL + s), TC_PRODUCERS);
-            mbar_init(bar(BAR_K_EMPTY + s), 2);      // one commit per Q tile
-            mbar_init(bar(BAR_V_EMPTY + s), 2);
+            mbar_init(bar(BAR_K_EMPTY + s), 1);
+            mbar_init(bar(BAR_V_EMPTY + s), 1);
             mbar_init(bar(BAR_S_READY + s), 1);
-            mbar_init(bar(BAR_O_READY + s), 1);
+            mbar_init(bar(BAR_P_READY + s), 128);        // every softmax thread of the tile arrives
+        }
+        for (int q = 0; q < 2; ++q) {
+            mbar_init(bar(BAR_PV_DONE + q), 1);
+            mbar_init(bar(BAR_O_READY + q), 1);
         }
         mbar_init_fence();
     }
@@ -190,14 +206,14 @@ attend_tc_kernel(TcAttendParams p) {
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
-    // columns: S of Q tile q at q * 128, O of Q tile q at 256 + q * D
-    if (warp < TC_SOFTMAX_WARPS) reg_alloc<TC_REGS_SOFTMAX>();
+    // columns: S of Q tile q, buffer u at q * 128 + u * 64; O of Q tile q at 256 + q * D
+    if (warp_u < TC_SOFTMAX_WARPS) reg_alloc<TC_REGS_SOFTMAX>();
     else reg_dealloc<TC_REGS_OTHER>();
 
-    if (warp < TC_SOFTMAX_WARPS) {
+    if (warp_u < TC_SOFTMAX_WARPS) {
         // ------------------------------------------------------------ softmax, one row per thread
-        const int qt = warp >> 2;                        // Q tile of this warpgroup
-        const int lane_base = (warp & 3) * 32;           // TMEM lanes this warp may touch
+        const int qt = warp_u >> 2;                      // Q tile of this warpgroup
+        const int lane_base = (warp_u & 3) * 32;         // TMEM lanes this warp may touch
         const int row = row0 + qt * 128 + lane_base + lane;
         const uint32_t tS = tmem_addr(tmem, lane_base, qt * 128);
         const uint32_t tO = tmem_addr(tmem, lane_base, 256 + qt * D);
@@ -206,61 +222,32 @@ attend_tc_kernel(TcAttendParams p) {
         const float sl2 = p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
 
-        // ---- MMA issue: lane 0 of the group's first warp
-        const bool issuer = (warp & 3) == 0 && lane == 0;
-        constexpr uint32_t ID_QK = idesc_bf16(128, TC_BN, false, false);
-        constexpr uint32_t ID_PV = idesc_bf16(128, D, false, true);
-        const uint32_t hi = desc_hi_sw128();
-        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)) + qt * (TILE_BYTES >> 4);
-        const uint32_t klo = desc_lo_kmajor(smem_u32(sK)), vlo = desc_lo_mnmajor(smem_u32(sV), BLK_BYTES);
-        const uint32_t dS = tmem + qt * 128, dO = tmem + 256 + qt * D;
-        // descriptor low words advance by compile-time constants (bytes >> 4)
-        auto issue_qk = [&](int s) {
-            const uint32_t b0 = klo + s * (TILE_BYTES >> 4);
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t o = ((ks >> 2) * BLK_BYTES + (ks & 3) * 32) >> 4;
-                umma_ss(dS, qlo + o, b0 + o, hi, ID_QK, ks);
-            }
-        };
-        auto issue_pv = [&](int s, int acc) {
-            const uint32_t b0 = vlo + s * (TILE_BYTES >> 4);
-#pragma unroll
-            for (int ks = 0; ks < TC_BN / 16; ++ks) umma_ts(dO, dS + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks);
-        };
-        if (issuer && n_tiles > 0) {
-            mbar_wait(bar(BAR_Q_FULL), 0, wc);
-            mbar_wait(bar(BAR_K_FULL + 0), 0, wc);
-            fence_async_smem();
-            tc_fence_after_sync();
-            issue_qk(0);
-            umma_commit(bar(BAR_S_READY + qt));
-            umma_commit(bar(BAR_K_EMPTY + 0));
-        }
-        __syncwarp();
-
         for (int j = 0; j < n_tiles; ++j) {
             const int key0 = (tile_begin + j) * TC_BN;
-            mbar_wait(bar(BAR_S_READY + qt), j & 1, wc);
+            const int u = j & 1;
+            mbar_wait(bar(BAR_S_READY + qt * 2 + u), (j >> 1) & 1, wc);
             tc_fence_after_sync();
             const bool need_mask = key0 + TC_BN > lim_min;
-            // the whole score row of this thread: 128 fp32 columns
+            // the score row of this thread: 64 fp32 columns
             uint32_t v[TC_BN];
-#pragma unroll
-            for (int c0 = 0; c0 < TC_BN; c0 += 32) tmem_ld32(tS + c0, v + c0);
+            tmem_ld32(tS + u * 64, v);
+            tmem_ld32(tS + u * 64 + 32, v + 32);
             tmem_wait_ld();
             if (need_mask) {
 #pragma unroll
                 for (int i = 0; i < TC_BN; ++i)
                     if (key0 + i >= lim) v[i] = 0xff800000u;     // -inf
             }
-            float mx0 = -INFINITY, mx1 = -INFINITY;
+            float mxc[8];
 #pragma unroll
-            for (int i = 0; i < TC_BN; i += 4) {
-                mx0 = fmax3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-                mx1 = fmax3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-            }
-            const float m_new = fmaxf(m_run, fmaxf(mx0, mx1) * sl2);
+            for (int c = 0; c < 8; ++c) mxc[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+#pragma unroll
+            for (int i = 16; i < TC_BN; i += 16)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    mxc[c] = fmax3(mxc[c], __uint_as_float(v[i + 2 * c]), __uint_as_float(v[i + 2 * c + 1]));
+            const float mx = fmaxf(fmax3(mxc[0], mxc[1], mxc[2]), fmax3(fmax3(mxc[3], mxc[4], mxc[5]), mxc[6], mxc[7]));
+            const float m_new = fmaxf(m_run, mx * sl2);
             const bool grow = m_new > m_run + kRescaleThreshold;
             if (__any_sync(0xffffffffu, grow)) {
                 // 0 on a row's first visible tile; a row that has seen no key yet keeps (m, l) = (-inf, 0)
@@ -268,7 +255,9 @@ attend_tc_kernel(TcAttendParams p) {
                 l_run *= alpha;
                 m_run = m_new;
                 if (j > 0) {
-                    // the commit that made S ready also covers the previous P V product: O is quiescent
+                    // O must be quiescent: wait for the P V product of the previous tile
+                    mbar_wait(bar(BAR_PV_DONE + qt), (j - 1) & 1, wc);
+                    tc_fence_after_sync();
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 32) {
                         uint32_t o[32];
@@ -280,56 +269,38 @@ attend_tc_kernel(TcAttendParams p) {
                     }
                 }
             }
-            // P = 2^(S * scale - m) as packed bf16 over the first half of the S columns.
+            // P = 2^(S * scale - m) as packed bf16 over the first half of the S buffer.
             // A row without a visible key so far has m = -inf: its P must be 0, not 2^(+inf).
             const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
             const float2 sl2v = make_float2(sl2, sl2), nm = make_float2(neg_m, neg_m);
-            float2 sum2 = make_float2(0.f, 0.f);
+            float2 sum4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            uint32_t pk[TC_BN / 2];
 #pragma unroll
-            for (int c0 = 0; c0 < TC_BN; c0 += 32) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float2 x = ffma2(make_float2(__uint_as_float(v[c0 + 2 * i]), __uint_as_float(v[c0 + 2 * i + 1])),
-                                           sl2v, nm);
-                    float2 e;
-                    if ((i & 3) < TC_POLY_PAIRS_OF_4) {
-                        e = exp2_poly2(x);
-                    } else {
-                        e.x = fast_exp2(x.x);
-                        e.y = fast_exp2(x.y);
-                    }
-                    sum2 = fadd2(sum2, e);
-                    pk[i] = pack_bf16(e.x, e.y);
+            for (int i = 0; i < TC_BN / 2; ++i) {
+                const float2 x = ffma2(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2v, nm);
+                float2 e;
+                if ((i & 3) < TC_POLY_PAIRS_OF_4) {
+                    e = exp2_poly2(x);
+                } else {
+                    e.x = fast_exp2(x.x);
+                    e.y = fast_exp2(x.y);
                 }
-                tmem_st16(tS + (c0 >> 1), pk);
+                sum4[i & 3] = fadd2(sum4[i & 3], e);
+                pk[i] = pack_bf16(e.x, e.y);
             }
-            l_run += sum2.x + sum2.y;
+            tmem_st32(tS + u * 64, pk);
+            {
+                const float2 a = fadd2(sum4[0], sum4[1]), c = fadd2(sum4[2], sum4[3]);
+                l_run += (a.x + a.y) + (c.x + c.y);
+            }
             tmem_wait_st();
             tc_fence_before_sync();
-            // every row of P is in tensor memory: named barrier over the 128 threads of the group
-            asm volatile("bar.sync %0, 128;\n" ::"r"(1 + qt) : "memory");
-            if (issuer) {
-                const int s = j & 1, sn = s ^ 1;
-                tc_fence_after_sync();
-                mbar_wait(bar(BAR_V_FULL + s), (j >> 1) & 1, wc);
-                fence_async_smem();
-                issue_pv(s, j > 0);
-                umma_commit(bar(BAR_V_EMPTY + s));
-                if (j + 1 < n_tiles) {
-                    mbar_wait(bar(BAR_K_FULL + sn), ((j + 1) >> 1) & 1, wc);
-                    fence_async_smem();
-                    issue_qk(sn);                      // overwrites S (and P) after the P V product, in issue order
-                    umma_commit(bar(BAR_S_READY + qt));
-                    umma_commit(bar(BAR_K_EMPTY + sn));
-                } else {
-                    umma_commit(bar(BAR_O_READY + qt));
-                }
-            }
-            __syncwarp();
+            mbar_arrive(bar(BAR_P_READY + qt * 2 + u));
         }
 
         // ---- epilogue: O / l  (or the unnormalised partial for the split merge)
+        // (BAR_PV_DONE cannot serve here: a parity wait tells adjacent phases apart only, and this
+        // thread may be two phases behind or level with it; BAR_O_READY completes exactly once.)
         if (n_tiles > 0) {
             mbar_wait(bar(BAR_O_READY + qt), 0, wc);
             tc_fence_after_sync();
@@ -341,18 +312,18 @@ attend_tc_kernel(TcAttendParams p) {
             __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(tO + c0, v);
+                uint32_t o[32];
+                tmem_ld32(tO + c0, o);
                 tmem_wait_ld();
                 if (row_ok) {
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(v[q4 * 8 + 0]) * inv, __uint_as_float(v[q4 * 8 + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(v[q4 * 8 + 2]) * inv, __uint_as_float(v[q4 * 8 + 3]) * inv);
-                        o.z = pack_bf16(__uint_as_float(v[q4 * 8 + 4]) * inv, __uint_as_float(v[q4 * 8 + 5]) * inv);
-                        o.w = pack_bf16(__uint_as_float(v[q4 * 8 + 6]) * inv, __uint_as_float(v[q4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(dst + c0 + q4 * 8) = o;
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(o[q4 * 8 + 0]) * inv, __uint_as_float(o[q4 * 8 + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(o[q4 * 8 + 2]) * inv, __uint_as_float(o[q4 * 8 + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(o[q4 * 8 + 4]) * inv, __uint_as_float(o[q4 * 8 + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(o[q4 * 8 + 6]) * inv, __uint_as_float(o[q4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(dst + c0 + q4 * 8) = w;
                     }
                 }
             }
@@ -361,14 +332,14 @@ attend_tc_kernel(TcAttendParams p) {
             if (n_tiles > 0) {
 #pragma unroll
                 for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tO + c0, v);
+                    uint32_t o[32];
+                    tmem_ld32(tO + c0, o);
                     tmem_wait_ld();
                     if (row_ok) {
 #pragma unroll
                         for (int i = 0; i < 32; i += 2)
                             *reinterpret_cast<float2*>(dst + c0 + i) =
-                                make_float2(__uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                                make_float2(__uint_as_float(o[i]), __uint_as_float(o[i + 1]));
                     }
                 }
             }
@@ -377,13 +348,12 @@ attend_tc_kernel(TcAttendParams p) {
                 dst[D + 1] = l_run;
             }
         }
-    } else {
+    } else if (warp_u < TC_MMA_WARP) {
         // ------------------------------------------------------------ producers: Q, then K/V tiles
         const int ptid = tid - TC_SOFTMAX_WARPS * 32;      // 0..127
         const int chunk = ptid % CH;                       // this thread's 16-byte chunk of every row
         const int rsub = ptid / CH;                        // first row handled
         constexpr int RSTEP = TC_PRODUCERS / CH;           // rows advanced per iteration
-        const uint32_t blk_off = (chunk >> 3) * BLK_BYTES; // 64-column block of the chunk
         const int cin = chunk & 7;
         if (n_tiles > 0) {
             for (int r = rsub; r < TC_ROWS; r += RSTEP) {
@@ -392,7 +362,7 @@ attend_tc_kernel(TcAttendParams p) {
                 const int cq = ok ? row / G : 0, g = ok ? row % G : 0;
                 const __nv_bfloat16* src = p.Q + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + chunk * 8;
                 const int rr = r & 127;
-                uint8_t* dst = sQ + (r >> 7) * TILE_BYTES + blk_off + rr * 128 + ((cin ^ (rr & 7)) << 4);
+                uint8_t* dst = sQ + (r >> 7) * Q_TILE_BYTES + (chunk >> 3) * Q_BLK_BYTES + rr * 128 + ((cin ^ (rr & 7)) << 4);
                 cp_async16(dst, src, ok ? 16 : 0);
             }
             cp_async_arrive_noinc(bar(BAR_Q_FULL));
@@ -401,11 +371,11 @@ attend_tc_kernel(TcAttendParams p) {
         const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
+        const uint32_t blk_off = (chunk >> 3) * KV_BLK_BYTES;
         for (int j = 0; j < n_tiles; ++j) {
-            const int s = j & 1;
-            const uint32_t ph = ((j >> 1) & 1) ^ 1;
+            const int s = j % TC_STAGES;
+            const uint32_t ph = ((j / TC_STAGES) & 1) ^ 1;
             const int key0 = (tile_begin + j) * TC_BN;
-            // positions of this thread's rows
             int pos[TC_BN / RSTEP];
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
@@ -420,7 +390,7 @@ attend_tc_kernel(TcAttendParams p) {
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int r = rsub + it * RSTEP;
-                uint8_t* dst = sK + s * TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
+                uint8_t* dst = sK + s * KV_TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
                 cp_async16(dst, Kb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
             }
             cp_async_arrive_noinc(bar(BAR_K_FULL + s));
@@ -428,12 +398,67 @@ attend_tc_kernel(TcAttendParams p) {
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int r = rsub + it * RSTEP;
-                uint8_t* dst = sV + s * TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
+                uint8_t* dst = sV + s * KV_TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
                 cp_async16(dst, Vb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
             }
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
         }
         cp_async_wait<0>();
+    } else if (warp_u == TC_MMA_WARP && n_tiles > 0) {
+        // ------------------------------------------------------------ MMA issue: converged warp, lane 0 leads
+        const uint32_t lead = lane == 0;
+        constexpr uint32_t ID_QK = idesc_bf16(128, TC_BN, false, false);
+        constexpr uint32_t ID_PV = idesc_bf16(128, D, false, true);
+        const uint32_t hi = desc_hi_sw128();
+        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)), klo = desc_lo_kmajor(smem_u32(sK));
+        const uint32_t vlo = desc_lo_mnmajor(smem_u32(sV), KV_BLK_BYTES);
+        // descriptor low words advance by compile-time constants (bytes >> 4)
+        auto issue_qk = [&](int qt, int s, int u) {         // S[qt][u] = Q[qt] . K[s]^T
+            const uint32_t a0 = qlo + qt * (Q_TILE_BYTES >> 4), b0 = klo + s * (KV_TILE_BYTES >> 4);
+            const uint32_t d = tmem + qt * 128 + u * 64;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks)
+                umma_ss(d, a0 + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
+                        b0 + (((ks >> 2) * KV_BLK_BYTES + (ks & 3) * 32) >> 4), hi, ID_QK, ks, lead);
+        };
+        auto issue_pv = [&](int qt, int s, int u, int acc) { // O[qt] (+)= P[qt][u] . V[s]
+            const uint32_t b0 = vlo + s * (KV_TILE_BYTES >> 4);
+            const uint32_t d = tmem + 256 + qt * D, a = tmem + qt * 128 + u * 64;
+#pragma unroll
+            for (int ks = 0; ks < TC_BN / 16; ++ks) umma_ts(d, a + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks, lead);
+        };
+        mbar_wait(bar(BAR_Q_FULL), 0, wc);
+        for (int j = 0; j < 2 && j < n_tiles; ++j) {          // scores of the first two tiles
+            mbar_wait(bar(BAR_K_FULL + j), 0, wc);
+            fence_async_smem();
+            tc_fence_after_sync();
+            for (int qt = 0; qt < 2; ++qt) {
+                issue_qk(qt, j, j);
+                umma_commit(bar(BAR_S_READY + qt * 2 + j), lead);
+            }
+            umma_commit(bar(BAR_K_EMPTY + j), lead);
+        }
+        for (int j = 0; j < n_tiles; ++j) {
+            const int s = j % TC_STAGES, u = j & 1;
+            const int jn = j + 2, sn = jn % TC_STAGES;
+            const bool more = jn < n_tiles;
+            mbar_wait(bar(BAR_V_FULL + s), (j / TC_STAGES) & 1, wc);
+            if (more) mbar_wait(bar(BAR_K_FULL + sn), (jn / TC_STAGES) & 1, wc);
+            fence_async_smem();
+            for (int qt = 0; qt < 2; ++qt) {
+                mbar_wait(bar(BAR_P_READY + qt * 2 + u), (j >> 1) & 1, wc);
+                tc_fence_after_sync();
+                issue_pv(qt, s, u, j > 0);
+                umma_commit(bar(BAR_PV_DONE + qt), lead);
+                if (j + 1 == n_tiles) umma_commit(bar(BAR_O_READY + qt), lead);
+                if (qt == 1) umma_commit(bar(BAR_V_EMPTY + s), lead);
+                if (more) {
+                    issue_qk(qt, sn, u);      // reuses buffer u after the P V product above, in issue order
+                    umma_commit(bar(BAR_S_READY + qt * 2 + u), lead);
+                    if (qt == 1) umma_commit(bar(BAR_K_EMPTY + sn), lead);
+                }
+            }
+        }
     }
 
     tc_fence_before_sync();
@@ -447,7 +472,7 @@ template <int D>
 static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_max, cudaStream_t st, int* nsplit_out) {
     const int R = p.l_C * p.G;
     const int row_tiles = (R + TC_ROWS - 1) / TC_ROWS;
-    constexpr int smem = 6 * TC_BN * D * 2 + 1024;
+    constexpr int smem = 2 * 128 * D * 2 + 2 * TC_STAGES * TC_BN * D * 2 + 1024;
     cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     // the in-kernel register split assumes the launch allocation it was sized for

@@ -186,40 +186,53 @@ __device__ __forceinline__ uint32_t desc_lo_mnmajor(uint32_t smem_byte_addr, uin
     return ((smem_byte_addr & 0x3ffff) >> 4) | ((lbo_bytes >> 4) << 16);
 }
 
-// D[tmem] (+)= A[smem] . B[smem]; one thread issues.  accumulate = 0 overwrites D.
+// The issue helpers below are meant to be called by a whole, converged warp: every lane
+// computes the (warp-uniform) operands, which lets the compiler keep them in uniform
+// registers, and only the lane whose `lead` is non-zero executes the instruction.  The
+// same lane must lead every MMA and every commit that tracks them.
+//
+// D[tmem] (+)= A[smem] . B[smem].  accumulate = 0 overwrites D.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                        uint32_t accumulate) {
+                                        uint32_t accumulate, uint32_t lead) {
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         ".reg .b64 da, db;\n"
         "setp.ne.b32 p, %5, 0;\n"
+        "setp.ne.b32 q, %6, 0;\n"
         "mov.b64 da, {%1, %3};\n"
         "mov.b64 db, {%2, %3};\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n"
         "}\n" ::"r"(d_tmem),
-        "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(lead)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] . B[smem].  A: row i of the tile in lane i, reduction elements 2c and
 // 2c+1 packed (low, high half) in column c.
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
-                                        uint32_t accumulate) {
+                                        uint32_t accumulate, uint32_t lead) {
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         ".reg .b64 db;\n"
         "setp.ne.b32 p, %5, 0;\n"
+        "setp.ne.b32 q, %6, 0;\n"
         "mov.b64 db, {%2, %3};\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n"
         "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(lead)
         : "memory");
 }
-// The mbarrier receives one arrival when every tcgen05.mma issued so far by this thread is done.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar)
-                 : "memory");
+// The mbarrier receives one arrival when every tcgen05.mma issued so far by the leading lane is done.
+__device__ __forceinline__ void umma_commit(uint32_t bar, uint32_t lead) {
+    asm volatile(
+        "{\n"
+        ".reg .pred q;\n"
+        "setp.ne.b32 q, %1, 0;\n"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+        "}\n" ::"r"(bar),
+        "r"(lead)
+        : "memory");
 }
 
 // ------------------------------------------------------------------ TMA
