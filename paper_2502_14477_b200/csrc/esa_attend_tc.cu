@@ -17,7 +17,7 @@
 //   * Warp roles: warps 0-3 / 4-7 run the online softmax of Q tile 0 / 1 (one thread per
 //     row holding its 64 scores in registers, so row maxima and sums need no shuffles),
 //     warps 8-11 gather K/V rows with index-driven 16-byte cp.async into 128-byte-swizzled
-//     tiles, warp 12 issues every MMA.  The issuing warp runs converged (all lanes compute
+//     tiles, warps 12 and 13 issue the MMAs of Q tile 0 and 1.  An issuing warp runs converged (all lanes compute
 //     the warp-uniform descriptors, lane 0 executes the tcgen05 instructions): a single
 //     diverged thread was starved of issue slots by the arithmetic-heavy softmax warps that
 //     share its scheduler (measured 100-600 cycles per tcgen05.mma instead of 64).
@@ -190,8 +190,8 @@ attend_tc_kernel(TcAttendParams p) {
         for (int s = 0; s < TC_STAGES; ++s) {
             mbar_init(bar(BAR_K_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_V_FULL + s), TC_PRODUCERS);
-            mbar_init(bar(BAR_K_EMPTY + s), 1);
-            mbar_init(bar(BAR_V_EMPTY + s), 1);
+            mbar_init(bar(BAR_K_EMPTY + s), 2);          // one commit per Q tile's issuing warp
+            mbar_init(bar(BAR_V_EMPTY + s), 2);
             mbar_init(bar(BAR_S_READY + s), 1);
             mbar_init(bar(BAR_P_READY + s), 128);        // every softmax thread of the tile arrives
         }
@@ -404,38 +404,40 @@ attend_tc_kernel(TcAttendParams p) {
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
         }
         cp_async_wait<0>();
-    } else if (warp_u == TC_MMA_WARP && n_tiles > 0) {
-        // ------------------------------------------------------------ MMA issue: converged warp, lane 0 leads
+    } else if (warp_u < TC_MMA_WARP + 2 && n_tiles > 0) {
+        // ------------------------------------------------------------ MMA issue: one converged warp per Q tile,
+        // lane 0 leads.  Two warps halve the chain of waits and commits that sits between batches of MMAs
+        // (the tensor core's queue is too shallow to hide it); their products interleave freely because the
+        // Q tiles share nothing but read-only K/V tiles.
+        const int qt = warp_u - TC_MMA_WARP;
         const uint32_t lead = lane == 0;
         constexpr uint32_t ID_QK = idesc_bf16(128, TC_BN, false, false);
         constexpr uint32_t ID_PV = idesc_bf16(128, D, false, true);
         const uint32_t hi = desc_hi_sw128();
-        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)), klo = desc_lo_kmajor(smem_u32(sK));
-        const uint32_t vlo = desc_lo_mnmajor(smem_u32(sV), KV_BLK_BYTES);
+        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)) + qt * (Q_TILE_BYTES >> 4);
+        const uint32_t klo = desc_lo_kmajor(smem_u32(sK)), vlo = desc_lo_mnmajor(smem_u32(sV), KV_BLK_BYTES);
+        const uint32_t dS = tmem + qt * 128, dO = tmem + 256 + qt * D;
         // descriptor low words advance by compile-time constants (bytes >> 4)
-        auto issue_qk = [&](int qt, int s, int u) {         // S[qt][u] = Q[qt] . K[s]^T
-            const uint32_t a0 = qlo + qt * (Q_TILE_BYTES >> 4), b0 = klo + s * (KV_TILE_BYTES >> 4);
-            const uint32_t d = tmem + qt * 128 + u * 64;
+        auto issue_qk = [&](int s, int u) {                 // S[u] = Q . K[s]^T
+            const uint32_t b0 = klo + s * (KV_TILE_BYTES >> 4);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
-                umma_ss(d, a0 + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
+                umma_ss(dS + u * 64, qlo + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
                         b0 + (((ks >> 2) * KV_BLK_BYTES + (ks & 3) * 32) >> 4), hi, ID_QK, ks, lead);
         };
-        auto issue_pv = [&](int qt, int s, int u, int acc) { // O[qt] (+)= P[qt][u] . V[s]
+        auto issue_pv = [&](int s, int u, int acc) {         // O (+)= P[u] . V[s]
             const uint32_t b0 = vlo + s * (KV_TILE_BYTES >> 4);
-            const uint32_t d = tmem + 256 + qt * D, a = tmem + qt * 128 + u * 64;
 #pragma unroll
-            for (int ks = 0; ks < TC_BN / 16; ++ks) umma_ts(d, a + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks, lead);
+            for (int ks = 0; ks < TC_BN / 16; ++ks)
+                umma_ts(dO, dS + u * 64 + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks, lead);
         };
         mbar_wait(bar(BAR_Q_FULL), 0, wc);
         for (int j = 0; j < 2 && j < n_tiles; ++j) {          // scores of the first two tiles
             mbar_wait(bar(BAR_K_FULL + j), 0, wc);
             fence_async_smem();
             tc_fence_after_sync();
-            for (int qt = 0; qt < 2; ++qt) {
-                issue_qk(qt, j, j);
-                umma_commit(bar(BAR_S_READY + qt * 2 + j), lead);
-            }
+            issue_qk(j, j);
+            umma_commit(bar(BAR_S_READY + qt * 2 + j), lead);
             umma_commit(bar(BAR_K_EMPTY + j), lead);
         }
         for (int j = 0; j < n_tiles; ++j) {
@@ -445,18 +447,16 @@ attend_tc_kernel(TcAttendParams p) {
             mbar_wait(bar(BAR_V_FULL + s), (j / TC_STAGES) & 1, wc);
             if (more) mbar_wait(bar(BAR_K_FULL + sn), (jn / TC_STAGES) & 1, wc);
             fence_async_smem();
-            for (int qt = 0; qt < 2; ++qt) {
-                mbar_wait(bar(BAR_P_READY + qt * 2 + u), (j >> 1) & 1, wc);
-                tc_fence_after_sync();
-                issue_pv(qt, s, u, j > 0);
-                umma_commit(bar(BAR_PV_DONE + qt), lead);
-                if (j + 1 == n_tiles) umma_commit(bar(BAR_O_READY + qt), lead);
-                if (qt == 1) umma_commit(bar(BAR_V_EMPTY + s), lead);
-                if (more) {
-                    issue_qk(qt, sn, u);      // reuses buffer u after the P V product above, in issue order
-                    umma_commit(bar(BAR_S_READY + qt * 2 + u), lead);
-                    if (qt == 1) umma_commit(bar(BAR_K_EMPTY + sn), lead);
-                }
+            mbar_wait(bar(BAR_P_READY + qt * 2 + u), (j >> 1) & 1, wc);
+            tc_fence_after_sync();
+            issue_pv(s, u, j > 0);
+            umma_commit(bar(BAR_PV_DONE + qt), lead);
+            if (j + 1 == n_tiles) umma_commit(bar(BAR_O_READY + qt), lead);
+            umma_commit(bar(BAR_V_EMPTY + s), lead);
+            if (more) {
+                issue_qk(sn, u);              // reuses buffer u after the P V product above, in issue order
+                umma_commit(bar(BAR_S_READY + qt * 2 + u), lead);
+                umma_commit(bar(BAR_K_EMPTY + sn), lead);
             }
         }
     }

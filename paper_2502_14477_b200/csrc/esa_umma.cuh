@@ -48,7 +48,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Every wait is bounded.  When a wait runs out (about a second), the thread records
+// try_wait with a suspend-time hint: the hardware parks the warp until the phase completes or
+// the hint (nanoseconds) runs out, so a waiting warp does not compete for issue slots with the
+// warps that are doing arithmetic or issuing MMAs on the same scheduler.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+
+// Every wait is bounded.  When a wait runs out (about two seconds), the thread records
 // ESA_ERR_TIMEOUT (5) in the device status word and raises the CTA-wide abort flag; from
 // then on every wait of the CTA returns at once, so the kernel drains, frees its tensor
 // memory and exits with wrong data but a usable context.
@@ -57,14 +74,13 @@ struct WaitCtx {
     int* status;                // global status word
 };
 constexpr long long kWaitLimitCycles = 4000000000LL;
+constexpr uint32_t kParkNs = 20000;     // one parked try_wait lasts at most this long
 
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (true) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return;
+        if (mbar_try_wait_parked(bar, parity, kParkNs)) return;
         if (*w.abort_flag) return;
         if (clock64() - t0 > kWaitLimitCycles) {
             *w.abort_flag = 1;
