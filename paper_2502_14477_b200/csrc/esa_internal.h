@@ -59,6 +59,11 @@ cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int row
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
                          const SeqMeta& meta, int max_lM, cudaStream_t st);
 
+// The same for chunks of >= 64 queries and d' in {64, 128} on tcgen05 with TMA-fed tiles; expects
+// ctx->rkey and ctx->skey zeroed.  cudaErrorNotSupported when the shape is not covered.
+cudaError_t launch_score_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
+                            const SeqMeta& meta, int max_lM, cudaStream_t st);
+
 // Eq. 8 + Eq. 2 on ctx->skey -> idx_out / n_sel_out.
 cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM,
                           int32_t* idx_out, int32_t* n_sel_out, cudaStream_t st);

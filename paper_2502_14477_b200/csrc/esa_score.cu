@@ -281,6 +281,12 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
     e = cudaMemset2DAsync(ctx->skey, sizeof(uint32_t) * ctx->cfg.max_tokens, 0,
                           sizeof(uint32_t) * (size_t)max_lM, B, st);
     if (e != cudaSuccess) return e;
+    // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels
+    if (l_C >= 64 && (DC == 64 || DC == 128) && (int64_t)B * ctx->cfg.max_tokens < (int64_t(1) << 31)) {
+        e = launch_score_tc(ctx, B, l_C, kc_cache, meta, max_lM, st);
+        if (e != cudaErrorNotSupported) return e;
+        cudaGetLastError();
+    }
     ScoreParams p;
     p.kc = kc_cache; p.qc = ctx->Qc; p.rkey = ctx->rkey; p.skey = ctx->skey;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.meta = meta;
