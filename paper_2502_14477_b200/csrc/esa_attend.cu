@@ -261,29 +261,43 @@ attend_kernel(AttendParams p) {
 
 // Merge of the split-KV partials (Algorithm 1's merge generalised to nsplit parts):
 // O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with M = max_s m_s.
+// One warp per output row: each lane owns D / 32 consecutive columns, so a part's row is one
+// coalesced read and the result one coalesced bf16 write.
 template <int D>
-__global__ void attend_merge_kernel(AttendParams p) {
+__global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
+    constexpr int PER = D / 32;                  // columns per lane: 2 or 4
     const int R = p.l_C * p.G;
-    const int row = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    if (row >= R) return;
     const float* base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit * R + row) * (D + 2);
     const int64_t sstride = (int64_t)R * (D + 2);
     float M = -INFINITY;
-    for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, base[s * sstride + D]);
+    for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, __ldg(base + s * sstride + D));
     float den = 0.f;
+    float acc[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
     for (int s = 0; s < p.nsplit; ++s) {
-        float m = base[s * sstride + D];
-        if (m > -INFINITY) den += fast_exp2(m - M) * base[s * sstride + D + 1];
-    }
-    const int cq = row / p.G, g = row % p.G;
-    __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * p.G + g) * D;
-    for (int col = threadIdx.x; col < D; col += blockDim.x) {
-        float acc = 0.f;
-        for (int s = 0; s < p.nsplit; ++s) {
-            float m = base[s * sstride + D];
-            if (m > -INFINITY) acc += fast_exp2(m - M) * base[s * sstride + col];
+        const float* ps = base + s * sstride;
+        const float m = __ldg(ps + D);
+        if (m == -INFINITY) continue;            // an empty part (uniform over the warp)
+        const float w = fast_exp2(m - M);
+        den += w * __ldg(ps + D + 1);
+        // rows start at multiples of (D + 2) floats: 8-byte aligned, so read pairs
+#pragma unroll
+        for (int i = 0; i < PER; i += 2) {
+            const float2 v = __ldg(reinterpret_cast<const float2*>(ps + lane * PER + i));
+            acc[i] += w * v.x;
+            acc[i + 1] += w * v.y;
         }
-        dst[col] = __float2bfloat16_rn(acc / den);
     }
+    const float inv = 1.f / den;
+    const int cq = row / p.G, g = row % p.G;
+    __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * p.G + g) * D + lane * PER;
+#pragma unroll
+    for (int i = 0; i < PER; i += 2) *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
 }
 
 template <int D, int NW, int BN>
@@ -312,7 +326,7 @@ static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     attend_kernel<D, NW, BN><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
     ctx->launches += 1;
     if (nsplit > 1) {
-        attend_merge_kernel<D><<<dim3(R, p.HG, B), D / 2, 0, st>>>(p);
+        attend_merge_kernel<D><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
         ctx->launches += 1;
     }
     return cudaGetLastError();
@@ -341,8 +355,8 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
         if (e != cudaSuccess) return e;
         if (nsplit > 1) {
             p.nsplit = nsplit;
-            if (ctx->d == 128) attend_merge_kernel<128><<<dim3(R, p.HG, B), 64, 0, st>>>(p);
-            else attend_merge_kernel<64><<<dim3(R, p.HG, B), 32, 0, st>>>(p);
+            if (ctx->d == 128) attend_merge_kernel<128><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
+            else attend_merge_kernel<64><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
             ctx->launches += 1;
         }
         return cudaGetLastError();
