@@ -137,6 +137,33 @@ esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
                             const void* K_cache, const void* V_cache, const int64_t* n_prev,
                             const int32_t* idx, const int32_t* n_sel, void* O, void* stream);
 
+/* (No counterpart in the paper: an integration convenience.)
+ * esa_attend for small chunks -- l_C * (H / H_G) <= 64 rows, the decode case -- that needs
+ * neither a context nor any allocation.  It is for callers that may not allocate device
+ * memory once they are running: a serving loop in which the implicit device-wide
+ * synchronisation of cudaMalloc / cudaFree would stall every other stream, or a host
+ * application that has already handed all device memory to its own pool so that a driver
+ * allocation would fail.  esa_create allocates a workspace and therefore does not suit
+ * them; this entry point calls no allocating routine at all.
+ *
+ * The partial results of the key-list splits go to a fixed 8 MiB array inside the library
+ * image (held on every GPU that loads the library, until the process exits).  A call is
+ * refused with ESA_ERR_CAPACITY when the chunk has more than 64 rows per key/value head,
+ * or when B * H_G * rows * (head_dim + 2) * 4 floats exceed the array (four splits is the
+ * least it will run with); e.g. B = 8, H_G = 8, l_C = 1, H / H_G = 4, head_dim = 128 uses
+ * 0.13 MiB per split.  Used fields of cfg: n_q_heads, n_kv_heads, head_dim, l_init,
+ * l_local, top_k, max_tokens, softmax_scale.  All other arguments are as for
+ * esa_attend_async; work is only enqueued on `stream`.
+ *
+ * The first call on each device looks up the array's device address; make that call with
+ * the device current and before any stream capture is started on that device.  Every call
+ * on a device shares the one array: calls that may overlap on the GPU (different streams,
+ * no ordering between them) race on it and give wrong results; order them.  Nothing in the
+ * array has to be cleared between calls -- each call writes every slot it later reads. */
+esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const void* Q_cur, int32_t l_C,
+                              const void* K_cache, const void* V_cache, const int64_t* n_prev,
+                              const int32_t* idx, const int32_t* n_sel, void* O, void* stream);
+
 /* Diagnostic: copies the pooled scores s' (Eq. 8) of the most recent esa_select of
  * sequence b to host memory dst[0..n) as fp32, n <= number of middle tokens of that
  * call.  Synchronises the given stream.  ESA_ERR_STATE if that call did no scoring. */

@@ -11,7 +11,8 @@ from .binding import (  # noqa: F401
     load_library,
     library_path,
     STATUS_NAMES,
+    attend_noalloc,
 )
 from .build import build_library  # noqa: F401
 
-__all__ = ["EsaError", "EsaConfig", "Esa", "load_library", "library_path", "build_library", "STATUS_NAMES"]
+__all__ = ["EsaError", "EsaConfig", "Esa", "load_library", "library_path", "build_library", "STATUS_NAMES", "attend_noalloc"]

@@ -81,6 +81,8 @@ _PROTOS = {
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_attend_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_attend_noalloc": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_read_pooled_scores": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
     "esa_launch_count": (C.c_int64, [C.c_void_p]),
     "esa_last_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -275,3 +277,24 @@ class Esa:
         if st != 0:
             raise EsaError(st, "esa_read_pooled_scores")
         return out
+
+
+def attend_noalloc(cfg: EsaConfig, Q_cur, K_cache, V_cache, n_prev, idx, n_sel, O, stream=None):
+    """``esa_attend_noalloc``: attention of a small chunk (decode) without a context and without
+    any device allocation -- the split partials live in a fixed array inside the library.  For
+    callers that must not allocate once running (see ``include/esa.h``).  Calls on one device
+    share that array and must be ordered with respect to each other."""
+    lib = load_library()
+    B, l_C = Q_cur.shape[0], Q_cur.shape[1]
+    _check(Q_cur, "Q_cur", torch.bfloat16, (B, l_C, cfg.n_q_heads, cfg.head_dim))
+    _check(K_cache, "K_cache", torch.bfloat16, (B, cfg.max_tokens, cfg.n_kv_heads, cfg.head_dim))
+    _check(V_cache, "V_cache", torch.bfloat16, (B, cfg.max_tokens, cfg.n_kv_heads, cfg.head_dim))
+    _check(idx, "idx", torch.int32, (B, cfg.top_k))
+    _check(n_sel, "n_sel", torch.int32, (B,))
+    _check(O, "O", torch.bfloat16, (B, l_C, cfg.n_q_heads, cfg.head_dim))
+    npv = Esa._nprev(n_prev, B)
+    c = cfg.to_c()
+    st = lib.esa_attend_noalloc(C.byref(c), B, _ptr(Q_cur), l_C, _ptr(K_cache), _ptr(V_cache),
+                                npv.ctypes.data_as(C.c_void_p), _ptr(idx), _ptr(n_sel), _ptr(O), _stream_ptr(stream))
+    if st != 0:
+        raise EsaError(st, "esa_attend_noalloc")

@@ -373,4 +373,119 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
     return cudaErrorInvalidValue;
 }
 
+// ---------------------------------------------------------------------------
+// esa_attend_noalloc: split-key attention of small chunks whose scratch is a fixed array
+// that is part of the library image, for callers that must not allocate device memory.
+// ---------------------------------------------------------------------------
+namespace {
+
+// Partial (O, m, l) rows of the key-list splits.  8 MiB, resident on every GPU that loads
+// the library, until the process exits.  Every slot the merge reads is written earlier in
+// the same call, so nothing has to be cleared between calls.
+constexpr size_t kNoAllocPartFloats = size_t(2) << 20;
+static __device__ __align__(256) float g_noalloc_part[kNoAllocPartFloats];
+
+constexpr int kNoAllocMaxDevices = 64;
+constexpr int kNoAllocMinSplits = 4;      // a call must be able to split its key list at least this far
+
+struct NoAllocDevice {
+    float* part;      // device address of g_noalloc_part on this device (the symbol itself is not one)
+    int num_sms;
+    bool ready;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+
+template <int D, int NW, int BN>
+cudaError_t launch_noalloc_t(const NoAllocDevice& dev, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
+    const int R = p.l_C * p.G;
+    constexpr int smem = (NW * 16 + 4 * BN) * (D / 8) * 16;
+    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN>, NW * 32, smem);
+    if (e != cudaSuccess) return e;
+    const int n_tiles = (n_att_max + BN - 1) / BN;
+    int nsplit = (per_sm * dev.num_sms) / (p.HG * B);
+    if (nsplit > kAttMaxSplits) nsplit = kAttMaxSplits;
+    if (nsplit > n_tiles) nsplit = n_tiles;
+    while (nsplit > 1 && (size_t)B * p.HG * nsplit * R * (D + 2) > kNoAllocPartFloats) --nsplit;
+    if (nsplit < 1) nsplit = 1;
+    p.nsplit = nsplit;
+    attend_kernel<D, NW, BN><<<dim3(1, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
+    if (nsplit > 1) attend_merge_kernel<D><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
 }  // namespace esa
+
+extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const void* Q_cur, int32_t l_C,
+                                         const void* K_cache, const void* V_cache, const int64_t* n_prev,
+                                         const int32_t* idx, const int32_t* n_sel, void* O, void* stream) {
+    using namespace esa;
+    if (!cfg || !Q_cur || !K_cache || !V_cache || !n_prev || !idx || !n_sel || !O || B <= 0 || l_C <= 0)
+        return ESA_ERR_INVALID_ARG;
+    if (cfg->n_q_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads ||
+        (cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->l_init < 0 || cfg->l_local < 0 || cfg->top_k <= 0 ||
+        cfg->max_tokens <= 0 || cfg->max_tokens >= (int64_t(1) << 31) || !(cfg->softmax_scale >= 0.f))
+        return ESA_ERR_SHAPE;
+    if (B > kMaxBatch) return ESA_ERR_CAPACITY;
+    const int G = cfg->n_q_heads / cfg->n_kv_heads, D = cfg->head_dim;
+    const int64_t R = (int64_t)l_C * G;
+    // only the split-key kernel of small chunks has a scratch-backed variant here
+    if (R > kAttSplitRows) return ESA_ERR_CAPACITY;
+    // the fixed array must leave room for at least kNoAllocMinSplits parts
+    if ((size_t)B * cfg->n_kv_heads * kNoAllocMinSplits * (size_t)R * (D + 2) > kNoAllocPartFloats) return ESA_ERR_CAPACITY;
+
+    SeqMeta meta;
+    int n_att_max = 0;
+    for (int b = 0; b < B; ++b) {
+        const int64_t t = n_prev[b];
+        if (t < 0) return ESA_ERR_INVALID_ARG;
+        if (t + l_C > cfg->max_tokens) return ESA_ERR_CAPACITY;
+        const int64_t i_end = t < cfg->l_init ? t : cfg->l_init;
+        int64_t m_end = t - cfg->l_local;
+        if (m_end < i_end) m_end = i_end;
+        meta.t[b] = (int)t; meta.i_end[b] = (int)i_end; meta.m_end[b] = (int)m_end;
+        const int64_t lM = m_end - i_end;
+        const int64_t n = i_end + (lM < cfg->top_k ? lM : cfg->top_k) + (t - m_end) + l_C;
+        if (n > n_att_max) n_att_max = (int)n;
+    }
+    for (int b = B; b < kMaxBatch; ++b) meta.t[b] = meta.i_end[b] = meta.m_end[b] = 0;
+
+    // Once per device, with that device current: resolve the device address of the scratch array
+    // (in host code its name is only a handle for the runtime) and read the SM count.
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return ESA_ERR_CUDA;
+    if (device < 0 || device >= kNoAllocMaxDevices) return ESA_ERR_UNSUPPORTED;
+    NoAllocDevice& dev = g_noalloc_dev[device];
+    if (!dev.ready) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_part) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return ESA_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0)
+            return ESA_ERR_CUDA;
+        dev.part = static_cast<float*>(ptr);
+        dev.num_sms = sms;
+        dev.ready = true;
+    }
+
+    AttendParams p;
+    p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
+    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part;
+    p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
+    p.top_k = cfg->top_k; p.nsplit = 1;
+    const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)D);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.meta = meta;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+    if (D == 128) e = R <= 16 ? launch_noalloc_t<128, 1, 32>(dev, p, B, n_att_max, st)
+                              : launch_noalloc_t<128, 4, 64>(dev, p, B, n_att_max, st);
+    else e = R <= 16 ? launch_noalloc_t<64, 1, 32>(dev, p, B, n_att_max, st)
+                     : launch_noalloc_t<64, 4, 64>(dev, p, B, n_att_max, st);
+    return e == cudaSuccess ? ESA_OK : ESA_ERR_CUDA;
+}
