@@ -132,6 +132,7 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->dH = c->H * c->d; c->dG = c->HG * c->d; c->G = c->H / c->HG;
     c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)c->d);
     c->has_w = c->has_bq = c->has_bk = false;
+    c->has_wmaps = false;
     c->launches = 0;
     c->last_scored = false;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
@@ -188,6 +189,9 @@ esa_status esa_set_compressors(esa_ctx* ctx, const float* Wq, const float* bq, c
     ctx->has_bk = bk != nullptr;
     if (bq && cudaMemcpy(ctx->bq, bq, 4 * ctx->dc, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
     if (bk && cudaMemcpy(ctx->bk, bk, 4 * ctx->dc, cudaMemcpyHostToDevice) != cudaSuccess) return ESA_ERR_CUDA;
+    ctx->has_wmaps = (ctx->dc == 64 || ctx->dc == 128) && ctx->dH % 128 == 0 && ctx->dG % 128 == 0 &&
+                     make_tensor_map_bf16(&ctx->wq_map, ctx->Wq, (uint64_t)ctx->dc, (uint64_t)ctx->dH, (uint32_t)ctx->dc) &&
+                     make_tensor_map_bf16(&ctx->wk_map, ctx->Wk, (uint64_t)ctx->dc, (uint64_t)ctx->dG, (uint32_t)ctx->dc);
     ctx->has_w = true;
     return ESA_OK;
 }
@@ -233,6 +237,13 @@ esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, i
         map.row0[b] = (int)n_prev[b];
     }
     if (n_new == 0) return ESA_OK;
+    if (ctx->has_wmaps) {
+        cudaError_t e = launch_compress_tc(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, &ctx->wk_map,
+                                           ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
+                                           ctx->cfg.max_tokens, map, (cudaStream_t)stream);
+        if (e != cudaErrorNotSupported) return from_cuda(e);
+        cudaGetLastError();
+    }
     return from_cuda(launch_compress(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, ctx->Wk,
                                      ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
                                      ctx->cfg.max_tokens, map, (cudaStream_t)stream));
@@ -274,8 +285,15 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     // q' = f_q(q) (Eq. 5)
     RowMap zero;
     for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
-    e = launch_compress(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
-                        ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, st);
+    e = cudaErrorNotSupported;
+    if (ctx->has_wmaps)
+        e = launch_compress_tc(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, &ctx->wq_map,
+                               ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, st);
+    if (e == cudaErrorNotSupported) {
+        cudaGetLastError();
+        e = launch_compress(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
+                            ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, st);
+    }
     if (e != cudaSuccess) return ESA_ERR_CUDA;
     // sequences that select everything need no scores: give them an empty middle part
     SeqMeta smeta = meta;

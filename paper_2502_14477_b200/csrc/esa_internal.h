@@ -1,6 +1,7 @@
 // Host-side declarations shared by the translation units of the ESA library.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -33,6 +34,8 @@ struct esa_ctx {
     bool has_w, has_bq, has_bk;
     __nv_bfloat16* Wq;   // [dc, dH]
     __nv_bfloat16* Wk;   // [dc, dG]
+    CUtensorMap wq_map, wk_map;   // TMA descriptors of Wq / Wk (valid when has_wmaps)
+    bool has_wmaps;
     float* bq;           // [dc]
     float* bk;           // [dc]
     __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
@@ -84,6 +87,17 @@ cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* 
                              const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
                              const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
                              int n_att_max, cudaStream_t st, int* nsplit_out);
+
+// TMA descriptor of a row-major bf16 matrix [rows, cols] (cols a multiple of 64), read in boxes of
+// box_rows x 64 columns with the 128-byte swizzle.  False when the driver entry point is missing
+// or refuses the shape.
+bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+// Eq. 5 on tcgen05 for d' in {64, 128} and d_in a multiple of 128.  X is [rows, d_in] contiguous.
+// cudaErrorNotSupported when the shape is not covered (the caller then uses the mma.sync kernel).
+cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
+                               const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
+                               int64_t dst_seq_stride, const RowMap& map, cudaStream_t st);
 
 cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new,
                              const __nv_bfloat16* V_new, int n_new, __nv_bfloat16* K_cache,

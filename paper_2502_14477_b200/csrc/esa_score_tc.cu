@@ -224,45 +224,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver entry point is looked up at run time so that the library carries no link-time
-// dependency on libcuda.
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-// rows x dc bf16, row-major; boxes of 128 rows x 64 columns in the 128-byte swizzle
-bool make_map(CUtensorMap* map, const void* base, uint64_t rows, int dc) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)dc, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)dc * 2};
-    cuuint32_t box[2] = {64, 128};
-    cuuint32_t es[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int DC>
 cudaError_t launch_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache, const SeqMeta& meta, int max_lM,
                      cudaStream_t st) {
     CUtensorMap kmap, qmap;
-    if (!make_map(&kmap, kc_cache, (uint64_t)B * ctx->cfg.max_tokens, DC)) return cudaErrorNotSupported;
-    if (!make_map(&qmap, ctx->Qc, (uint64_t)B * l_C, DC)) return cudaErrorNotSupported;
+    if (!make_tensor_map_bf16(&kmap, kc_cache, (uint64_t)B * ctx->cfg.max_tokens, DC, 128)) return cudaErrorNotSupported;
+    if (!make_tensor_map_bf16(&qmap, ctx->Qc, (uint64_t)B * l_C, DC, 128)) return cudaErrorNotSupported;
     ScoreTcParams p;
     p.rkey = ctx->rkey; p.skey = ctx->skey; p.status = ctx->status;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.meta = meta;
