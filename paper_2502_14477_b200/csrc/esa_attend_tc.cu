@@ -30,6 +30,8 @@
 //     or the split merge, needs no correction.
 //   * A long key list can be split across CTAs (blockIdx.z); partial (O, m, l) go to the
 //     context's scratch and the merge kernel of esa_attend.cu combines them.
+#include <cstring>
+
 #include "esa_internal.h"
 #include "esa_umma.cuh"
 
@@ -68,6 +70,7 @@ struct TcAttendParams {
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
+    int q_tma;          // Q tiles arrive by TMA (one arrival) instead of cp.async (one per producer thread)
     float scale_log2;
     SeqMeta meta;
 };
@@ -141,7 +144,7 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
 
 template <int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-attend_tc_kernel(TcAttendParams p) {
+attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     constexpr int CH = D / 8;                   // 16-byte chunks per row
     constexpr int Q_TILE_BYTES = 128 * D * 2;   // one 128-row Q tile
     constexpr int Q_BLK_BYTES = 128 * 128;      // one 64-column block of it
@@ -186,7 +189,7 @@ attend_tc_kernel(TcAttendParams p) {
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar(BAR_Q_FULL), TC_PRODUCERS);
+        mbar_init(bar(BAR_Q_FULL), p.q_tma ? 1 : TC_PRODUCERS);
         for (int s = 0; s < TC_STAGES; ++s) {
             mbar_init(bar(BAR_K_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_V_FULL + s), TC_PRODUCERS);
@@ -355,7 +358,19 @@ attend_tc_kernel(TcAttendParams p) {
         const int rsub = ptid / CH;                        // first row handled
         constexpr int RSTEP = TC_PRODUCERS / CH;           // rows advanced per iteration
         const int cin = chunk & 7;
-        if (n_tiles > 0) {
+        if (n_tiles > 0 && p.q_tma) {
+            // two boxes per 64-column block: rows (query, head-in-group) of one key/value head
+            if (ptid == 0) {
+                mbar_arrive_expect_tx(bar(BAR_Q_FULL), 2 * Q_TILE_BYTES);
+#pragma unroll
+                for (int qt = 0; qt < 2; ++qt)
+#pragma unroll
+                    for (int blk = 0; blk < D / 64; ++blk)
+                        tma_load_3d(smem_u32(sQ + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), &qmap, blk * 64, kvh * G,
+                                    b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
+            }
+        } else if (n_tiles > 0) {
+            // group sizes that do not divide 128: 16-byte copies, row by row
             for (int r = rsub; r < TC_ROWS; r += RSTEP) {
                 const int row = row0 + r;
                 const bool ok = row < R;
@@ -499,7 +514,10 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     }
     p.nsplit = best;
     *nsplit_out = best;
-    attend_tc_kernel<D><<<dim3(row_tiles, p.HG, B * best), TC_THREADS, smem, st>>>(p);
+    CUtensorMap qmap;
+    p.q_tma = make_tensor_map_q(&qmap, p.Q, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
+    if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
+    attend_tc_kernel<D><<<dim3(row_tiles, p.HG, B * best), TC_THREADS, smem, st>>>(qmap, p);
     ctx->launches += 1;
     return cudaGetLastError();
 }

@@ -251,6 +251,20 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uin
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Q as a 3-D tensor [B * l_C, H, D] read in boxes of (128 / G queries) x (G heads) x 64 columns: the rows
+// of a box land in shared memory in (query, head-in-group) order, 128 bytes each, 128-byte swizzled.
+bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, int H, int D, int G) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || G <= 0 || 128 % G || D % 64 || (reinterpret_cast<uintptr_t>(base) & 15)) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)n_queries};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
+    cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G)};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
                                int64_t dst_seq_stride, const RowMap& map, cudaStream_t st) {

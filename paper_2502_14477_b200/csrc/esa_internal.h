@@ -93,6 +93,10 @@ cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* 
 // or refuses the shape.
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
+// TMA descriptor of the query tensor [n_queries, H, D] for the attention kernel (group size G must
+// divide 128).
+bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, int H, int D, int G);
+
 // Eq. 5 on tcgen05 for d' in {64, 128} and d_in a multiple of 128.  X is [rows, d_in] contiguous.
 // cudaErrorNotSupported when the shape is not covered (the caller then uses the mma.sync kernel).
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
