@@ -106,7 +106,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "200",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -191,23 +191,48 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
             attend_events.append((t, l_C, e0, e1))
 
 
-def run_prefill_layer_e2e(ctx, cfg, L, bufs, caches, stage, O_host):
-    """Same work with HOST inputs and outputs: every chunk's Q/K/V rows are copied from
-    pinned host memory, appended to the device caches, and the chunk's output is copied back."""
+def run_prefill_layer_e2e(ctx, cfg, L, bufs, caches, stage, O_host, streams):
+    """Same work with HOST inputs and outputs: every chunk's Q/K/V rows are copied from pinned host
+    memory, appended to the device caches, and the chunk's output is copied back to pinned host
+    memory.  The copies run on their own streams through two sets of staging buffers, so the
+    transfer of chunk i+1 and the read-back of chunk i-1 overlap the kernels of chunk i; the
+    library calls are enqueued on the compute stream (the caller's stream, as any user would)."""
     Kc, idx, n_sel, _ = bufs
     Kcache, Vcache = caches
-    Qs, Ks, Vs, Os = stage
     hq, hk, hv = L.host
-    for t in range(0, cfg.S, cfg.l_C):
+    s_in, s_cmp, s_out = streams
+    cur = torch.cuda.current_stream()
+    for s in streams:
+        s.wait_stream(cur)
+    in_done = [torch.cuda.Event() for _ in range(2)]
+    cmp_done = [torch.cuda.Event() for _ in range(2)]
+    out_done = [torch.cuda.Event() for _ in range(2)]
+    for i, t in enumerate(range(0, cfg.S, cfg.l_C)):
         l_C = min(cfg.l_C, cfg.S - t)
-        Qs[0, :l_C].copy_(hq[t: t + l_C], non_blocking=True)
-        Ks[0, :l_C].copy_(hk[t: t + l_C], non_blocking=True)
-        Vs[0, :l_C].copy_(hv[t: t + l_C], non_blocking=True)
-        ctx.append_kv(Ks[:, :l_C], Vs[:, :l_C], Kcache, Vcache, [t])
-        ctx.compress_keys(Ks[:, :l_C], Kc, [t])
-        ctx.select(Qs[:, :l_C], Kc, [t], idx, n_sel)
-        ctx.attend(Qs[:, :l_C], Kcache, Vcache, [t], idx, n_sel, Os[:, :l_C])
-        O_host[t: t + l_C].copy_(Os[0, :l_C], non_blocking=True)
+        slot = i & 1
+        Qs, Ks, Vs, Os = stage[slot]
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(cmp_done[slot])          # the kernels of chunk i-2 have read this slot
+            Qs[0, :l_C].copy_(hq[t: t + l_C], non_blocking=True)
+            Ks[0, :l_C].copy_(hk[t: t + l_C], non_blocking=True)
+            Vs[0, :l_C].copy_(hv[t: t + l_C], non_blocking=True)
+            in_done[slot].record(s_in)
+        with torch.cuda.stream(s_cmp):
+            s_cmp.wait_event(in_done[slot])
+            if i >= 2:
+                s_cmp.wait_event(out_done[slot])         # chunk i-2's output has left this slot
+            ctx.append_kv(Ks[:, :l_C], Vs[:, :l_C], Kcache, Vcache, [t])
+            ctx.compress_keys(Ks[:, :l_C], Kc, [t])
+            ctx.select(Qs[:, :l_C], Kc, [t], idx, n_sel)
+            ctx.attend(Qs[:, :l_C], Kcache, Vcache, [t], idx, n_sel, Os[:, :l_C])
+            cmp_done[slot].record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(cmp_done[slot])
+            O_host[t: t + l_C].copy_(Os[0, :l_C], non_blocking=True)
+            out_done[slot].record(s_out)
+    for s in streams:
+        cur.wait_stream(s)
 
 
 # ----------------------------------------------------------------------------
@@ -384,7 +409,7 @@ def run_esa(args, cfg):
     att_ms = sum(a.elapsed_time(b) for (_, _, a, b) in events)
     att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
     achieved = att_flops / (att_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attend_kernel", "achieved": achieved, "peak": peaks["tflops_sustained"],
+    roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (+ attend_merge_kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": None,
                 "peak_source": peaks["source"] + " sustained bf16", "share_of_step": att_ms / (ms_total),
                 "launches": len(events)}
@@ -392,20 +417,21 @@ def run_esa(args, cfg):
     # end to end: host inputs and outputs
     L0 = layers[0]
     caches = (torch.zeros_like(L0.K), torch.zeros_like(L0.V))
-    stage = (torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"),
-             torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
-             torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
-             torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"))
+    stage = [(torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"),
+              torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
+              torch.empty(1, cfg.l_C, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda"),
+              torch.empty(1, cfg.l_C, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda")) for _ in range(2)]
+    streams = tuple(torch.cuda.Stream() for _ in range(3))
     O_host = torch.empty(cfg.S, cfg.H, cfg.d, dtype=torch.bfloat16).pin_memory()
     ctx.set_compressors(L0.wq, None, L0.wk, None)
-    run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host)
+    run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host, streams)
     sync_all()
     n_e2e = max(1, min(2, args.steps))
     t0 = torch.cuda.Event(enable_timing=True)
     t1 = torch.cuda.Event(enable_timing=True)
     t0.record()
     for _ in range(n_e2e):
-        run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host)
+        run_prefill_layer_e2e(ctx, cfg, L0, bufs, caches, stage, O_host, streams)
     t1.record()
     sync_all()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1), "cuda" if world > 1 else None) / n_e2e
@@ -413,7 +439,7 @@ def run_esa(args, cfg):
     d2h = cfg.S * cfg.d_H * 2
     e2e = {"value": world * cfg.S / (N_LAYERS_STACK * e2e_ms * 1e-3), "unit": "tokens/s",
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms}
-    del caches, stage, layers
+    del caches, stage, layers, streams
     ctx.close()
     torch.cuda.empty_cache()
 
@@ -454,7 +480,7 @@ def run_esa(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--steps", type=int, default=8)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="esa", choices=["esa", "reference"])
     ap.add_argument("--layers", type=int, default=3, help="distinct layers' data kept resident")

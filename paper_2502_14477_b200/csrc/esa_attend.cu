@@ -300,6 +300,282 @@ __global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
     for (int i = 0; i < PER; i += 2) *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
 }
 
+// ---------------------------------------------------------------------------
+// Decode (one query per sequence): the step is bound by reading the gathered K/V rows, and the
+// arithmetic per row (G dot products and G axpys of length D) fits the FMA pipe many times over,
+// so no tensor-core fragments (they would be three-quarters padding).  Every warp streams its
+// rows through a private ring of shared-memory stages filled by index-driven 16-byte cp.async
+// (DEC_STAGES - 1 stages of 4 KB in flight per warp, the positions looked up one iteration
+// further ahead), D / 8 lanes share a row, and every lane group runs its own online softmax over
+// the rows it saw; groups, warps and key-list splits are merged with the same (O, m, l)
+// algebra as Algorithm 1's merge.
+// ---------------------------------------------------------------------------
+constexpr int DEC_UN = 4;          // rows per lane group and stage
+constexpr int DEC_WARPS = 4;
+constexpr int DEC_STAGES = 4;
+
+template <int D, int G>
+__global__ void __launch_bounds__(DEC_WARPS * 32)
+attend_decode_kernel(AttendParams p) {
+    constexpr int LPR = D / 8;                 // lanes per row
+    constexpr int GROUPS = 32 / LPR;           // rows per warp load
+    constexpr int KEYS_PER_ITER = GROUPS * DEC_UN;
+    constexpr int STAGE_BYTES = 2 * KEYS_PER_ITER * D * 2;   // K rows then V rows
+    extern __shared__ uint4 dec_smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gi = lane / LPR, li = lane % LPR;
+    const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    uint8_t* ring = reinterpret_cast<uint8_t*>(dec_smem) + warp * (DEC_STAGES * STAGE_BYTES);
+
+    const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
+    int n_sel = p.n_sel[b];
+    n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
+    const int n_glob = i_end + n_sel;
+    const int n_att = n_glob + (t - m_end) + 1;            // the single query sees every listed key
+
+    // this CTA's part of the key list, in whole iterations of one warp
+    const int iters_all = (n_att + KEYS_PER_ITER - 1) / KEYS_PER_ITER;
+    const int per = (iters_all + p.nsplit - 1) / p.nsplit;
+    const int it_begin = split * per, it_end = min(iters_all, it_begin + per);
+
+    const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + li * 8;
+    const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + li * 8;
+    const int32_t* idx = p.idx + (int64_t)b * p.top_k;
+    const int64_t tok_stride = (int64_t)p.HG * D;
+
+    // list positions -> token positions of the rows of iteration `it` that this lane group loads
+    auto lookup = [&](int it, int (&pos)[DEC_UN]) {
+#pragma unroll
+        for (int u = 0; u < DEC_UN; ++u) {
+            const int j = it * KEYS_PER_ITER + u * GROUPS + gi;
+            int q = -1;
+            if (it < it_end && j < n_att) {
+                if (j < i_end) q = j;
+                else if (j < n_glob) q = __ldg(idx + (j - i_end));
+                else q = m_end + (j - n_glob);
+            }
+            pos[u] = q;
+        }
+    };
+    auto issue = [&](int stage, const int (&pos)[DEC_UN]) {
+        uint8_t* sk = ring + stage * STAGE_BYTES;
+        uint8_t* sv = sk + KEYS_PER_ITER * D * 2;
+#pragma unroll
+        for (int u = 0; u < DEC_UN; ++u) {
+            const int64_t off = (int64_t)(pos[u] < 0 ? 0 : pos[u]) * tok_stride;
+            const int o = ((u * GROUPS + gi) * LPR + li) * 16;
+            cp_async16(sk + o, Kb + off, pos[u] < 0 ? 0 : 16);
+            cp_async16(sv + o, Vb + off, pos[u] < 0 ? 0 : 16);
+        }
+    };
+
+    // this lane's 8 columns of the G query rows, pre-scaled into the exp2 domain
+    float q[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p.Q + ((int64_t)b * p.H + kvh * G + g) * D + li * 8);
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __bfloat1622float2(h[i]);
+            q[g][2 * i] = f.x * p.scale_log2;
+            q[g][2 * i + 1] = f.y * p.scale_log2;
+        }
+    }
+    float m[G], l[G], acc[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        m[g] = -INFINITY;
+        l[g] = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
+    }
+
+    // prologue: DEC_STAGES - 1 iterations in flight, positions of one more in registers
+    int pos_next[DEC_UN];
+    const int it0 = it_begin + warp;
+#pragma unroll
+    for (int s = 0; s < DEC_STAGES - 1; ++s) {
+        lookup(it0 + s * DEC_WARPS, pos_next);
+        issue(s, pos_next);
+        cp_async_commit();
+    }
+    lookup(it0 + (DEC_STAGES - 1) * DEC_WARPS, pos_next);
+
+    int n = 0;
+    for (int it = it0; it < it_end; it += DEC_WARPS, ++n) {
+        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next);
+        cp_async_commit();
+        lookup(it + DEC_STAGES * DEC_WARPS, pos_next);
+        cp_async_wait<DEC_STAGES - 1>();
+        __syncwarp();
+        const uint8_t* sk = ring + (n % DEC_STAGES) * STAGE_BYTES;
+        const uint8_t* sv = sk + KEYS_PER_ITER * D * 2;
+        bool ok[DEC_UN];
+        float sc[DEC_UN][G];
+#pragma unroll
+        for (int u = 0; u < DEC_UN; ++u) {
+            ok[u] = it * KEYS_PER_ITER + u * GROUPS + gi < n_att;
+            const uint4 kr = *reinterpret_cast<const uint4*>(sk + ((u * GROUPS + gi) * LPR + li) * 16);
+            float kf[8];
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&kr);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(h[i]);
+                kf[2 * i] = f.x;
+                kf[2 * i + 1] = f.y;
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float a = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a = fmaf(q[g][i], kf[i], a);
+                sc[u][g] = a;
+            }
+        }
+#pragma unroll
+        for (int o = LPR / 2; o >= 1; o >>= 1)
+#pragma unroll
+            for (int u = 0; u < DEC_UN; ++u)
+#pragma unroll
+                for (int g = 0; g < G; ++g) sc[u][g] += __shfl_xor_sync(0xffffffffu, sc[u][g], o);
+        // online softmax per head, then the value rows
+        float vf[DEC_UN][8];
+#pragma unroll
+        for (int u = 0; u < DEC_UN; ++u) {
+            const uint4 vr = *reinterpret_cast<const uint4*>(sv + ((u * GROUPS + gi) * LPR + li) * 16);
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&vr);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(h[i]);
+                vf[u][2 * i] = f.x;
+                vf[u][2 * i + 1] = f.y;
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float mx = -INFINITY;
+#pragma unroll
+            for (int u = 0; u < DEC_UN; ++u) mx = fmaxf(mx, ok[u] ? sc[u][g] : -INFINITY);
+            const float m_new = fmaxf(m[g], mx);
+            const float ms = (m_new == -INFINITY) ? 0.f : m_new;
+            const float alpha = fast_exp2(m[g] - ms);
+            m[g] = m_new;
+            float pw[DEC_UN], sum = 0.f;
+#pragma unroll
+            for (int u = 0; u < DEC_UN; ++u) {
+                pw[u] = ok[u] ? fast_exp2(sc[u][g] - ms) : 0.f;
+                sum += pw[u];
+            }
+            l[g] = l[g] * alpha + sum;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float a = acc[g][i] * alpha;
+#pragma unroll
+                for (int u = 0; u < DEC_UN; ++u) a = fmaf(pw[u], vf[u][i], a);
+                acc[g][i] = a;
+            }
+        }
+        __syncwarp();          // the stage is free for the copy issued next iteration
+    }
+    cp_async_wait<0>();
+
+    // merge the lane groups of the warp (same columns li, different rows)
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float m_o = __shfl_xor_sync(0xffffffffu, m[g], o);
+            const float l_o = __shfl_xor_sync(0xffffffffu, l[g], o);
+            const float m_new = fmaxf(m[g], m_o);
+            const float ms = (m_new == -INFINITY) ? 0.f : m_new;
+            const float a = fast_exp2(m[g] - ms), bsc = fast_exp2(m_o - ms);
+            l[g] = l[g] * a + l_o * bsc;
+            m[g] = m_new;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float v_o = __shfl_xor_sync(0xffffffffu, acc[g][i], o);
+                acc[g][i] = acc[g][i] * a + v_o * bsc;
+            }
+        }
+    }
+    // merge the warps through shared memory (the rings are idle now)
+    __syncthreads();
+    float* s_m = reinterpret_cast<float*>(dec_smem);          // [DEC_WARPS][G]
+    float* s_l = s_m + DEC_WARPS * G;                          // [DEC_WARPS][G]
+    float* s_acc = s_l + DEC_WARPS * G;                        // [DEC_WARPS][G][D]
+    if (gi == 0) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            if (li == 0) { s_m[warp * G + g] = m[g]; s_l[warp * G + g] = l[g]; }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) s_acc[(warp * G + g) * D + li * 8 + i] = acc[g][i];
+        }
+    }
+    __syncthreads();
+    // thread (g, column) combines the DEC_WARPS parts
+    for (int e = tid; e < G * D; e += DEC_WARPS * 32) {
+        const int g = e / D, col = e % D;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, s_m[w * G + g]);
+        const float Ms = (M == -INFINITY) ? 0.f : M;
+        float o = 0.f, lsum = 0.f;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) {
+            const float wgt = fast_exp2(s_m[w * G + g] - Ms);
+            o += wgt * s_acc[(w * G + g) * D + col];
+            lsum += wgt * s_l[w * G + g];
+        }
+        if (p.nsplit == 1) {
+            p.O[((int64_t)b * p.H + kvh * G + g) * D + col] = __float2bfloat16_rn(o / lsum);
+        } else {
+            float* dst = p.part + ((((int64_t)b * p.HG + kvh) * p.nsplit + split) * G + g) * (D + 2);
+            dst[col] = o;
+            if (col == 0) { dst[D] = M; dst[D + 1] = lsum; }
+        }
+    }
+}
+
+template <int D, int G>
+static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
+    constexpr int keys_per_iter = (32 / (D / 8)) * DEC_UN;
+    constexpr int smem = DEC_WARPS * DEC_STAGES * 2 * keys_per_iter * D * 2;
+    static_assert(smem >= (2 * DEC_WARPS * G + DEC_WARPS * G * D) * 4, "the warp merge reuses the rings");
+    cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_decode_kernel<D, G>, DEC_WARPS * 32, smem);
+    if (e != cudaSuccess) return e;
+    const int iters = (n_att_max + keys_per_iter - 1) / keys_per_iter;
+    // one wave of CTAs, each warp with at least a few iterations
+    int nsplit = (per_sm * ctx->num_sms) / (p.HG * B);
+    if (nsplit > kAttMaxSplits) nsplit = kAttMaxSplits;
+    if (nsplit > (iters + 4 * DEC_WARPS - 1) / (4 * DEC_WARPS)) nsplit = (iters + 4 * DEC_WARPS - 1) / (4 * DEC_WARPS);
+    while (nsplit > 1 && (size_t)B * p.HG * nsplit * G * (D + 2) > ctx->att_part_elems) --nsplit;
+    if (nsplit < 1) nsplit = 1;
+    p.nsplit = nsplit;
+    attend_decode_kernel<D, G><<<dim3(nsplit, p.HG, B), DEC_WARPS * 32, smem, st>>>(p);
+    ctx->launches += 1;
+    if (nsplit > 1) {
+        attend_merge_kernel<D><<<dim3((G + 7) / 8, p.HG, B), 256, 0, st>>>(p);
+        ctx->launches += 1;
+    }
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t launch_decode(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
+    switch (p.G) {
+        case 1: return launch_decode_t<D, 1>(ctx, p, B, n_att_max, st);
+        case 2: return launch_decode_t<D, 2>(ctx, p, B, n_att_max, st);
+        case 4: return launch_decode_t<D, 4>(ctx, p, B, n_att_max, st);
+        case 7: return launch_decode_t<D, 7>(ctx, p, B, n_att_max, st);
+        case 8: return launch_decode_t<D, 8>(ctx, p, B, n_att_max, st);
+    }
+    return cudaErrorNotSupported;
+}
+
 template <int D, int NW, int BN>
 static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
     constexpr int BM = NW * 16;
@@ -360,6 +636,12 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
             ctx->launches += 1;
         }
         return cudaGetLastError();
+    }
+    if (l_C == 1) {
+        // decode: streaming kernel for the usual group sizes
+        cudaError_t e = ctx->d == 128 ? launch_decode<128>(ctx, p, B, n_att_max, st)
+                                      : launch_decode<64>(ctx, p, B, n_att_max, st);
+        if (e != cudaErrorNotSupported) return e;
     }
     if (ctx->d == 128) {
         if (R <= 16) return launch_attend_t<128, 1, 32>(ctx, p, B, n_att_max, st);
