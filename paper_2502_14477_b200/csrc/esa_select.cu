@@ -19,7 +19,7 @@ namespace cg = cooperative_groups;
 
 namespace esa {
 
-constexpr int SEL_CLUSTER = 8;
+constexpr int SEL_CLUSTER_MAX = 16;   // CTAs working on one sequence: 8, or 16 (beyond the portable size) for small batches
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_BINS = 2048;
 
@@ -103,10 +103,11 @@ __device__ __forceinline__ void find_bin(const uint32_t* g, int nb, uint32_t kre
     __syncthreads();
 }
 
-__global__ void __cluster_dims__(SEL_CLUSTER, 1, 1) __launch_bounds__(SEL_THREADS)
+__global__ void __launch_bounds__(SEL_THREADS)
 select_topk_kernel(SelectParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
+    const int n_ctas = (int)gridDim.x;          // = cluster size: one cluster per sequence
     const int b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -132,7 +133,7 @@ select_topk_kernel(SelectParams p) {
 
     // slice of this CTA: whole 32-element rows, contiguous
     const int rows32 = (l_M + 31) / 32;
-    const int rows_per_cta = (rows32 + SEL_CLUSTER - 1) / SEL_CLUSTER;
+    const int rows_per_cta = (rows32 + n_ctas - 1) / n_ctas;
     const int lo = min(l_M, rank * rows_per_cta * 32);
     const int hi = min(l_M, (rank + 1) * rows_per_cta * 32);
 
@@ -191,7 +192,7 @@ select_topk_kernel(SelectParams p) {
         for (int i = tid; i < nb; i += SEL_THREADS) {
             const uint32_t c = hist[i];
             if (c) {
-                for (int r = 0; r < SEL_CLUSTER; ++r) atomicAdd(cluster.map_shared_rank(&ghist[pass][i], r), c);
+                for (int r = 0; r < n_ctas; ++r) atomicAdd(cluster.map_shared_rank(&ghist[pass][i], r), c);
             }
         }
         cluster.sync();
@@ -302,15 +303,50 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.top_k = ctx->cfg.top_k; p.eps = ctx->cfg.eps;
     p.raw = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
+    cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    // 16 CTAs per sequence while the whole batch still fits the machine at once and the device can
+    // place such a cluster; else the portable 8
+    static int can16 = -1;
+    if (can16 < 0) {
+        cudaLaunchConfig_t probe = {};
+        probe.gridDim = dim3(SEL_CLUSTER_MAX, 1);
+        probe.blockDim = dim3(SEL_THREADS);
+        probe.dynamicSmemBytes = 0;
+        cudaLaunchAttribute pa[1];
+        pa[0].id = cudaLaunchAttributeClusterDimension;
+        pa[0].val.clusterDim.x = SEL_CLUSTER_MAX;
+        pa[0].val.clusterDim.y = 1;
+        pa[0].val.clusterDim.z = 1;
+        probe.attrs = pa;
+        probe.numAttrs = 1;
+        int n = 0;
+        can16 = (cudaOccupancyMaxActiveClusters(&n, select_topk_kernel, &probe) == cudaSuccess && n > 0) ? 1 : 0;
+        if (!can16) cudaGetLastError();
+    }
+    const int n_ctas = (can16 && B * SEL_CLUSTER_MAX <= ctx->num_sms / 2) ? SEL_CLUSTER_MAX : 8;
     // dynamic shared memory for a CTA's slice of pooled keys (largest sequence of the call)
     const int rows32 = (max_lM + 31) / 32;
-    const int slice = ((rows32 + SEL_CLUSTER - 1) / SEL_CLUSTER) * 32;
+    const int slice = ((rows32 + n_ctas - 1) / n_ctas) * 32;
     size_t smem = (size_t)slice * 4;
     if (smem > 160 * 1024) smem = 0;
     p.slice_cap = (int)(smem / 4);
-    cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ctas, B);
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = n_ctas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, select_topk_kernel, p);
     if (e != cudaSuccess) return e;
-    select_topk_kernel<<<dim3(SEL_CLUSTER, B), SEL_THREADS, smem, st>>>(p);
     ctx->launches += 1;
     return cudaGetLastError();
 }
