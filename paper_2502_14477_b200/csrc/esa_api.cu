@@ -240,7 +240,7 @@ esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, i
     if (ctx->has_wmaps) {
         cudaError_t e = launch_compress_tc(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, &ctx->wk_map,
                                            ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
-                                           ctx->cfg.max_tokens, map, (cudaStream_t)stream);
+                                           ctx->cfg.max_tokens, map, nullptr, 0, (cudaStream_t)stream);
         if (e != cudaErrorNotSupported) return from_cuda(e);
         cudaGetLastError();
     }
@@ -286,9 +286,13 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     RowMap zero;
     for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
     e = cudaErrorNotSupported;
-    if (ctx->has_wmaps)
+    bool rkey_cleared = false;
+    if (ctx->has_wmaps) {
+        // the compression kernel also clears the row-maximum words that the scoring pass accumulates into
         e = launch_compress_tc(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, &ctx->wq_map,
-                               ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, st);
+                               ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, ctx->rkey, B * l_C, st);
+        rkey_cleared = e == cudaSuccess;
+    }
     if (e == cudaErrorNotSupported) {
         cudaGetLastError();
         e = launch_compress(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
@@ -299,7 +303,7 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     SeqMeta smeta = meta;
     for (int b = 0; b < B; ++b)
         if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
-    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, st);
+    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, st);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
     e = launch_select(ctx, B, l_C, smeta, max_lM, idx_out, n_sel_out, st);
     return from_cuda(e);

@@ -273,24 +273,35 @@ __global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
     if (row >= R) return;
     const float* base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit * R + row) * (D + 2);
     const int64_t sstride = (int64_t)R * (D + 2);
+    // parts are taken four at a time so that their loads are in flight together
     float M = -INFINITY;
     for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, __ldg(base + s * sstride + D));
     float den = 0.f;
     float acc[PER];
 #pragma unroll
     for (int i = 0; i < PER; ++i) acc[i] = 0.f;
-    for (int s = 0; s < p.nsplit; ++s) {
-        const float* ps = base + s * sstride;
-        const float m = __ldg(ps + D);
-        if (m == -INFINITY) continue;            // an empty part (uniform over the warp)
-        const float w = fast_exp2(m - M);
-        den += w * __ldg(ps + D + 1);
-        // rows start at multiples of (D + 2) floats: 8-byte aligned, so read pairs
+    for (int s0 = 0; s0 < p.nsplit; s0 += 4) {
+        float mm[4], ll[4];
+        float2 v[4][PER / 2];
 #pragma unroll
-        for (int i = 0; i < PER; i += 2) {
-            const float2 v = __ldg(reinterpret_cast<const float2*>(ps + lane * PER + i));
-            acc[i] += w * v.x;
-            acc[i + 1] += w * v.y;
+        for (int j = 0; j < 4; ++j) {
+            const bool in = s0 + j < p.nsplit;
+            const float* ps = base + (in ? s0 + j : 0) * sstride;
+            mm[j] = in ? __ldg(ps + D) : -INFINITY;
+            ll[j] = __ldg(ps + D + 1);
+#pragma unroll
+            for (int i = 0; i < PER / 2; ++i) v[j][i] = __ldg(reinterpret_cast<const float2*>(ps + lane * PER + 2 * i));
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (mm[j] == -INFINITY) continue;        // an empty or absent part (uniform over the warp)
+            const float w = fast_exp2(mm[j] - M);
+            den += w * ll[j];
+#pragma unroll
+            for (int i = 0; i < PER / 2; ++i) {
+                acc[2 * i] += w * v[j][i].x;
+                acc[2 * i + 1] += w * v[j][i].y;
+            }
         }
     }
     const float inv = 1.f / den;

@@ -35,6 +35,8 @@ struct CompressTcParams {
     __nv_bfloat16* dst;
     int* status;
     int rows, rows_per_seq, kslice;
+    uint32_t* zero_words;      // optional: words the first CTA clears (the caller's next kernel accumulates there)
+    int zero_count;
     int64_t seq_stride;
     RowMap map;
 };
@@ -79,6 +81,8 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
 
+    if (p.zero_words && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = tid; i < p.zero_count; i += CT_THREADS) p.zero_words[i] = 0u;
     if (warp == 0) {
         if (lane == 0) {
             tma_prefetch_desc(&xmap);
@@ -142,10 +146,19 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         const int lr = split * band + i / PER_ROW, c4 = (i % PER_ROW) * 4;
         const int row = row0 + lr;
         if (row >= p.rows) continue;
+        // remote reads four at a time (their latencies overlap); the sum order stays split order
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp = 0; sp < nsplit; ++sp) {
-            const float4 v = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sPart, sp) + lr * PSTRIDE + c4);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        for (int sp0 = 0; sp0 < nsplit; sp0 += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                v[j] = sp0 + j < nsplit
+                           ? *reinterpret_cast<const float4*>(cluster.map_shared_rank(sPart, sp0 + j) + lr * PSTRIDE + c4)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                s.x += v[j].x; s.y += v[j].y; s.z += v[j].z; s.w += v[j].w;
+            }
         }
         if (p.bias) {
             s.x += p.bias[c4]; s.y += p.bias[c4 + 1]; s.z += p.bias[c4 + 2]; s.w += p.bias[c4 + 3];
@@ -160,7 +173,8 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
 
 template <int DC>
 cudaError_t launch_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_per_seq, int d_in, const CUtensorMap* wmap,
-                     const float* bias, __nv_bfloat16* dst, int64_t seq_stride, const RowMap& map, cudaStream_t st) {
+                     const float* bias, __nv_bfloat16* dst, int64_t seq_stride, const RowMap& map, uint32_t* zero_words,
+                     int zero_count, cudaStream_t st) {
     CUtensorMap xmap;
     if (!make_tensor_map_bf16(&xmap, X, (uint64_t)rows, (uint64_t)d_in, CT_ROWS)) return cudaErrorNotSupported;
     const int row_tiles = (rows + CT_ROWS - 1) / CT_ROWS;
@@ -200,6 +214,7 @@ cudaError_t launch_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_pe
     CompressTcParams p;
     p.bias = bias; p.dst = dst; p.status = ctx->status; p.rows = rows; p.rows_per_seq = rows_per_seq;
     p.kslice = d_in / nsplit; p.seq_stride = seq_stride; p.map = map;
+    p.zero_words = zero_words; p.zero_count = zero_count;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(row_tiles, nsplit);
     cfg.blockDim = dim3(CT_THREADS);
@@ -267,11 +282,12 @@ bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, i
 
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
-                               int64_t dst_seq_stride, const RowMap& map, cudaStream_t st) {
+                               int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
+                               cudaStream_t st) {
     if (d_in % CT_KCHUNK) return cudaErrorNotSupported;
     const int rows = B * rows_per_seq;
-    if (ctx->dc == 128) return launch_t<128>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, st);
-    if (ctx->dc == 64) return launch_t<64>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, st);
+    if (ctx->dc == 128) return launch_t<128>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st);
+    if (ctx->dc == 64) return launch_t<64>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st);
     return cudaErrorNotSupported;
 }
 

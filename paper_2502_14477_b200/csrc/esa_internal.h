@@ -59,11 +59,12 @@ cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int row
                             int64_t dst_seq_stride, const RowMap& map, cudaStream_t st);
 
 // Eq. 6 + Eq. 4: fills ctx->skey (and ctx->rkey) for the middle tokens of every sequence.
+// rkey_cleared: the caller's compression kernel has already zeroed ctx->rkey for this call.
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                         const SeqMeta& meta, int max_lM, cudaStream_t st);
+                         const SeqMeta& meta, int max_lM, bool rkey_cleared, cudaStream_t st);
 
 // The same for chunks of >= 64 queries and d' in {64, 128} on tcgen05 with TMA-fed tiles; expects
-// ctx->rkey and ctx->skey zeroed.  cudaErrorNotSupported when the shape is not covered.
+// ctx->rkey zeroed (pass 1 clears the part of ctx->skey that pass 2 accumulates into).  cudaErrorNotSupported when the shape is not covered.
 cudaError_t launch_score_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
                             const SeqMeta& meta, int max_lM, cudaStream_t st);
 
@@ -101,7 +102,14 @@ bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, i
 // cudaErrorNotSupported when the shape is not covered (the caller then uses the mma.sync kernel).
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
-                               int64_t dst_seq_stride, const RowMap& map, cudaStream_t st);
+                               int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
+                               cudaStream_t st);
+
+// True when launch_score takes the tcgen05 path for this call.
+inline bool score_uses_tc(const esa_ctx* ctx, int B, int l_C) {
+    return l_C >= 64 && (ctx->dc == 64 || ctx->dc == 128) &&
+           (int64_t)B * ctx->cfg.max_tokens < (int64_t(1) << 31);
+}
 
 cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new,
                              const __nv_bfloat16* V_new, int n_new, __nv_bfloat16* K_cache,

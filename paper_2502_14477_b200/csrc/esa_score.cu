@@ -261,8 +261,9 @@ score_decode_kernel(ScoreDecodeParams p) {
 
 template <int DC>
 static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                                  const SeqMeta& meta, int max_lM, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(ctx->rkey, 0, sizeof(uint32_t) * (size_t)B * l_C, st);
+                                  const SeqMeta& meta, int max_lM, bool rkey_cleared, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+    if (!rkey_cleared) e = cudaMemsetAsync(ctx->rkey, 0, sizeof(uint32_t) * (size_t)B * l_C, st);
     if (e != cudaSuccess) return e;
     if (l_C == 1) {
         ScoreDecodeParams p;
@@ -278,15 +279,15 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
         ctx->launches += 1;
         return cudaGetLastError();
     }
-    e = cudaMemset2DAsync(ctx->skey, sizeof(uint32_t) * ctx->cfg.max_tokens, 0,
-                          sizeof(uint32_t) * (size_t)max_lM, B, st);
-    if (e != cudaSuccess) return e;
-    // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels
-    if (l_C >= 64 && (DC == 64 || DC == 128) && (int64_t)B * ctx->cfg.max_tokens < (int64_t(1) << 31)) {
+    // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels (they clear skey themselves)
+    if (score_uses_tc(ctx, B, l_C)) {
         e = launch_score_tc(ctx, B, l_C, kc_cache, meta, max_lM, st);
         if (e != cudaErrorNotSupported) return e;
         cudaGetLastError();
     }
+    e = cudaMemset2DAsync(ctx->skey, sizeof(uint32_t) * ctx->cfg.max_tokens, 0,
+                          sizeof(uint32_t) * (size_t)max_lM, B, st);
+    if (e != cudaSuccess) return e;
     ScoreParams p;
     p.kc = kc_cache; p.qc = ctx->Qc; p.rkey = ctx->rkey; p.skey = ctx->skey;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.meta = meta;
@@ -308,11 +309,11 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
 }
 
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache, const SeqMeta& meta,
-                         int max_lM, cudaStream_t st) {
+                         int max_lM, bool rkey_cleared, cudaStream_t st) {
     switch (ctx->dc) {
-        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, st);
-        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, st);
-        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, st);
+        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
+        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
+        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -34,6 +34,7 @@ struct ScoreTcParams {
     int64_t max_tokens;
     int l_C;
     int combine;        // pass 2: more than one query block contributes to a key (atomic max)
+    int clear_skey;     // pass 1: the CTAs of query block 0 zero skey for the tiles they visit
     SeqMeta meta;
 };
 
@@ -165,6 +166,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
             if (PASS == 1) {
                 const int key0 = tile * ST_KEYS;
                 const bool tail = key0 + ST_KEYS > l_M;
+                if (p.clear_skey && blockIdx.y == 0 && key0 + et < l_M) p.skey[(int64_t)b * p.max_tokens + key0 + et] = 0u;
 #pragma unroll
                 for (int c0 = 0; c0 < ST_KEYS; c0 += 32) {
                     uint32_t v[32];
@@ -247,6 +249,7 @@ cudaError_t launch_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache
     };
     const int qb1 = (l_C + 127) / 128, qb2 = (l_C + 255) / 256;
     p.combine = 0;
+    p.clear_skey = qb2 > 1;
     score_tc_kernel<DC, 1><<<dim3(grid_x(qb1), qb1, B), ST_THREADS, smem1, st>>>(kmap, qmap, p);
     p.combine = qb2 > 1;
     score_tc_kernel<DC, 2><<<dim3(grid_x(qb2), qb2, B), ST_THREADS, smem2, st>>>(kmap, qmap, p);
@@ -256,8 +259,7 @@ cudaError_t launch_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache
 
 }  // namespace
 
-// Both scoring passes for chunks of at least 64 queries and d' of 64 or 128; rkey must be
-// zeroed and, when a chunk spans more than 256 queries, skey too (the caller does both).
+// Both scoring passes for chunks of at least 64 queries and d' of 64 or 128; rkey must be zeroed.
 // Returns cudaErrorNotSupported when this path does not cover the shape.
 cudaError_t launch_score_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache, const SeqMeta& meta,
                             int max_lM, cudaStream_t st) {
