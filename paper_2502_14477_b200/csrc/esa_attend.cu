@@ -266,6 +266,8 @@ attend_kernel(AttendParams p) {
 template <int D>
 __global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
     constexpr int PER = D / 32;                  // columns per lane: 2 or 4
+    pdl_wait();
+    pdl_launch_dependents();
     const int R = p.l_C * p.G;
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -337,6 +339,8 @@ attend_decode_kernel(AttendParams p) {
     const int gi = lane / LPR, li = lane % LPR;
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     uint8_t* ring = reinterpret_cast<uint8_t*>(dec_smem) + warp * (DEC_STAGES * STAGE_BYTES);
+    pdl_wait();
+    pdl_launch_dependents();
 
     const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
     int n_sel = p.n_sel[b];
@@ -566,13 +570,14 @@ static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     while (nsplit > 1 && (size_t)B * p.HG * nsplit * G * (D + 2) > ctx->att_part_elems) --nsplit;
     if (nsplit < 1) nsplit = 1;
     p.nsplit = nsplit;
-    attend_decode_kernel<D, G><<<dim3(nsplit, p.HG, B), DEC_WARPS * 32, smem, st>>>(p);
+    e = launch_pdl(attend_decode_kernel<D, G>, dim3(nsplit, p.HG, B), dim3(DEC_WARPS * 32), smem, st, p);
     ctx->launches += 1;
+    if (e != cudaSuccess) return e;
     if (nsplit > 1) {
-        attend_merge_kernel<D><<<dim3((G + 7) / 8, p.HG, B), 256, 0, st>>>(p);
+        e = launch_pdl(attend_merge_kernel<D>, dim3((G + 7) / 8, p.HG, B), dim3(256), 0, st, p);
         ctx->launches += 1;
     }
-    return cudaGetLastError();
+    return e;
 }
 
 template <int D>
@@ -642,11 +647,11 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
         if (e != cudaSuccess) return e;
         if (nsplit > 1) {
             p.nsplit = nsplit;
-            if (ctx->d == 128) attend_merge_kernel<128><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
-            else attend_merge_kernel<64><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
+            if (ctx->d == 128) e = launch_pdl(attend_merge_kernel<128>, dim3((R + 7) / 8, p.HG, B), dim3(256), 0, st, p);
+            else e = launch_pdl(attend_merge_kernel<64>, dim3((R + 7) / 8, p.HG, B), dim3(256), 0, st, p);
             ctx->launches += 1;
         }
-        return cudaGetLastError();
+        return e;
     }
     if (l_C == 1) {
         // decode: streaming kernel for the usual group sizes

@@ -169,21 +169,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     const int G = p.G;
     const int R = p.l_C * G;
 
-    const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
-    int n_sel = p.n_sel[b];
-    n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
-    const int n_glob = i_end + n_sel;
-    const int n_att = n_glob + (t - m_end) + p.l_C;
-    const int c_first = n_att - p.l_C;
-
-    const int r_last = min(R, row0 + TC_ROWS) - 1;
-    const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
-    const int n_tiles_all = (j_end + TC_BN - 1) / TC_BN;
-    const int per = (n_tiles_all + p.nsplit - 1) / p.nsplit;
-    const int tile_begin = split * per;
-    const int tile_end = min(n_tiles_all, tile_begin + per);
-    const int n_tiles = max(0, tile_end - tile_begin);
-
     WaitCtx wc{&abort_flag, p.status};
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
@@ -210,6 +195,24 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     // columns: S of Q tile q, buffer u at q * 128 + u * 64; O of Q tile q at 256 + q * D
+    // everything read from global memory comes after the preceding kernel (the selection) is complete
+    pdl_wait();
+    pdl_launch_dependents();
+    const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
+    int n_sel = p.n_sel[b];
+    n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
+    const int n_glob = i_end + n_sel;
+    const int n_att = n_glob + (t - m_end) + p.l_C;
+    const int c_first = n_att - p.l_C;
+
+    const int r_last = min(R, row0 + TC_ROWS) - 1;
+    const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
+    const int n_tiles_all = (j_end + TC_BN - 1) / TC_BN;
+    const int per = (n_tiles_all + p.nsplit - 1) / p.nsplit;
+    const int tile_begin = split * per;
+    const int tile_end = min(n_tiles_all, tile_begin + per);
+    const int n_tiles = max(0, tile_end - tile_begin);
+
     if (warp_u < TC_SOFTMAX_WARPS) reg_alloc<TC_REGS_SOFTMAX>();
     else reg_dealloc<TC_REGS_OTHER>();
 
@@ -517,9 +520,9 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     CUtensorMap qmap;
     p.q_tma = make_tensor_map_q(&qmap, p.Q, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
     if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
-    attend_tc_kernel<D><<<dim3(row_tiles, p.HG, B * best), TC_THREADS, smem, st>>>(qmap, p);
+    e = launch_pdl(attend_tc_kernel<D>, dim3(row_tiles, p.HG, B * best), dim3(TC_THREADS), smem, st, qmap, p);
     ctx->launches += 1;
-    return cudaGetLastError();
+    return e;
 }
 
 // Returns cudaErrorNotSupported when this path does not cover the shape (the caller then

@@ -82,6 +82,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// start while its predecessor in the stream is still draining.  pdl_wait() returns once the predecessor
+// has completed and its writes are visible (a no-op for an ordinary launch); everything a kernel
+// reads from or writes to global memory comes after it.  pdl_launch_dependents() lets the successor's
+// CTAs take the SMs this grid frees at its tail.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // 2^x, hardware approximation (ex2.approx: 2^-inf = +0)
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;

@@ -80,6 +80,8 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
 
     if (p.zero_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = tid; i < p.zero_count; i += CT_THREADS) p.zero_words[i] = 0u;
@@ -220,13 +222,15 @@ cudaError_t launch_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_pe
     cfg.blockDim = dim3(CT_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = nsplit;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     e = cudaLaunchKernelEx(&cfg, compress_tc_kernel<DC>, xmap, *wmap, p);
     ctx->launches += 1;
     return e;

@@ -11,6 +11,23 @@
 
 namespace esa {
 
+// Launch with the programmatic-serialization attribute (the kernel must call pdl_wait() before it
+// touches global memory).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int kAttMaxSplits = 64;     // split-KV factor of the attention kernel (small chunks)
 constexpr int kAttSplitRows = 64;     // split-KV is used only when l_C * (H/H_G) <= this
 constexpr int kAttPrefillSplits = 4; // largest split of a prefill-sized chunk's key list

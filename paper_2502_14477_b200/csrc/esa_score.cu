@@ -199,6 +199,8 @@ score_decode_kernel(ScoreDecodeParams p) {
     constexpr int LPR = DC / 8;         // lanes per key row (16 bytes each)
     constexpr int RPW = 32 / LPR;       // rows per warp access
     constexpr int UNROLL = 4;
+    pdl_wait();
+    pdl_launch_dependents();
     const int b = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int i_end = p.meta.i_end[b];
@@ -275,9 +277,9 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
         int cap = (8 * ctx->num_sms + B - 1) / B;
         if (gx > cap) gx = cap;
         if (gx < 1) gx = 1;
-        score_decode_kernel<DC><<<dim3(gx, B), 256, 0, st>>>(p);
+        e = launch_pdl(score_decode_kernel<DC>, dim3(gx, B), dim3(256), 0, st, p);
         ctx->launches += 1;
-        return cudaGetLastError();
+        return e;
     }
     // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels (they clear skey themselves)
     if (score_uses_tc(ctx, B, l_C)) {

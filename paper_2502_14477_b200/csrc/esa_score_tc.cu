@@ -96,6 +96,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();
+    pdl_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -250,9 +252,11 @@ cudaError_t launch_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache
     const int qb1 = (l_C + 127) / 128, qb2 = (l_C + 255) / 256;
     p.combine = 0;
     p.clear_skey = qb2 > 1;
-    score_tc_kernel<DC, 1><<<dim3(grid_x(qb1), qb1, B), ST_THREADS, smem1, st>>>(kmap, qmap, p);
+    e = launch_pdl(score_tc_kernel<DC, 1>, dim3(grid_x(qb1), qb1, B), dim3(ST_THREADS), smem1, st, kmap, qmap, p);
+    if (e != cudaSuccess) return e;
     p.combine = qb2 > 1;
-    score_tc_kernel<DC, 2><<<dim3(grid_x(qb2), qb2, B), ST_THREADS, smem2, st>>>(kmap, qmap, p);
+    e = launch_pdl(score_tc_kernel<DC, 2>, dim3(grid_x(qb2), qb2, B), dim3(ST_THREADS), smem2, st, kmap, qmap, p);
+    if (e != cudaSuccess) return e;
     ctx->launches += 2;
     return cudaGetLastError();
 }

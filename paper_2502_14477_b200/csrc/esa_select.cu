@@ -129,7 +129,6 @@ select_topk_kernel(SelectParams p) {
     const uint32_t* src = p.skey + (int64_t)b * p.max_tokens;
     uint32_t* pk = p.pkey + (int64_t)b * p.max_tokens;
     const int raw = p.raw;
-    const float r0 = raw ? key_to_f32(p.rkey[(int64_t)b * p.l_C]) : 0.f;
 
     // slice of this CTA: whole 32-element rows, contiguous
     const int rows32 = (l_M + 31) / 32;
@@ -142,6 +141,9 @@ select_topk_kernel(SelectParams p) {
         ghist[0][i] = ghist[1][i] = ghist[2][i] = 0;
     }
     cluster.sync();     // every CTA's histograms are zero before anyone adds to them remotely
+    pdl_wait();         // the scores come from the preceding kernel
+    pdl_launch_dependents();
+    const float r0 = raw ? key_to_f32(p.rkey[(int64_t)b * p.l_C]) : 0.f;
 
     // ---- digit 0: pool (Eq. 8), store pooled keys, histogram of bits 31..21
     // A warp loads 32 consecutive keys starting eps before its first output and slides the
@@ -338,13 +340,15 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     cfg.blockDim = dim3(SEL_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = n_ctas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     e = cudaLaunchKernelEx(&cfg, select_topk_kernel, p);
     if (e != cudaSuccess) return e;
     ctx->launches += 1;
