@@ -314,31 +314,32 @@ __global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
 }
 
 // ---------------------------------------------------------------------------
-// Decode (one query per sequence): the step is bound by reading the gathered K/V rows, and the
-// arithmetic per row (G dot products and G axpys of length D) fits the FMA pipe many times over,
-// so no tensor-core fragments (they would be three-quarters padding).  Every warp streams its
+// Decode (one query per sequence): the step is bound by reading the gathered K/V rows, so the
+// kernel is built around the stream of rows, not around the arithmetic.  Every warp pulls its
 // rows through a private ring of shared-memory stages filled by index-driven 16-byte cp.async
-// (DEC_STAGES - 1 stages of 4 KB in flight per warp, the positions looked up one iteration
-// further ahead), D / 8 lanes share a row, and every lane group runs its own online softmax over
-// the rows it saw; groups, warps and key-list splits are merged with the same (O, m, l)
-// algebra as Algorithm 1's merge.
+// (16 rows of K and of V per stage, DEC_STAGES - 1 stages in flight per warp, the positions
+// looked up one iteration further ahead).  The arithmetic runs on mma.sync with the rows on the
+// 16-wide M side -- S^T = K Q^T and O^T += V^T P^T -- so that the G <= 8 heads of the group sit
+// on the 8-wide N side: no padding along the long dimension and ~65 instructions per 16 rows.
+// Warps and key-list splits are merged with the (O, m, l) algebra of Algorithm 1's merge.
 // ---------------------------------------------------------------------------
-constexpr int DEC_UN = 4;          // rows per lane group and stage
 constexpr int DEC_WARPS = 4;
-constexpr int DEC_STAGES = 4;
+constexpr int DEC_STAGES = 3;
+constexpr int DEC_ROWS = 16;       // rows (keys) per stage
 
 template <int D, int G>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 attend_decode_kernel(AttendParams p) {
-    constexpr int LPR = D / 8;                 // lanes per row
-    constexpr int GROUPS = 32 / LPR;           // rows per warp load
-    constexpr int KEYS_PER_ITER = GROUPS * DEC_UN;
-    constexpr int STAGE_BYTES = 2 * KEYS_PER_ITER * D * 2;   // K rows then V rows
+    constexpr int CH = D / 8;                        // 16-byte chunks per row
+    constexpr int TILE_CHUNKS = DEC_ROWS * CH;       // one K or V tile, in chunks
+    constexpr int STAGE_CHUNKS = 2 * TILE_CHUNKS;
+    constexpr int PER_LANE = TILE_CHUNKS / 32;       // chunk copies per lane and tile
+    constexpr int ROWS_PER_PASS = 32 / CH;           // rows covered by one copy instruction of the warp
+    static_assert(G <= 8, "the heads of a group sit on the 8-wide side of the MMA");
     extern __shared__ uint4 dec_smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int gi = lane / LPR, li = lane % LPR;
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
-    uint8_t* ring = reinterpret_cast<uint8_t*>(dec_smem) + warp * (DEC_STAGES * STAGE_BYTES);
+    uint4* ring = dec_smem + warp * (DEC_STAGES * STAGE_CHUNKS);
     pdl_wait();
     pdl_launch_dependents();
 
@@ -349,65 +350,65 @@ attend_decode_kernel(AttendParams p) {
     const int n_att = n_glob + (t - m_end) + 1;            // the single query sees every listed key
 
     // this CTA's part of the key list, in whole iterations of one warp
-    const int iters_all = (n_att + KEYS_PER_ITER - 1) / KEYS_PER_ITER;
+    const int iters_all = (n_att + DEC_ROWS - 1) / DEC_ROWS;
     const int per = (iters_all + p.nsplit - 1) / p.nsplit;
     const int it_begin = split * per, it_end = min(iters_all, it_begin + per);
 
-    const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + li * 8;
-    const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + li * 8;
+    const int my_chunk = lane % CH, my_row = lane / CH;     // copies of this lane: rows my_row + i * ROWS_PER_PASS
+    const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
+    const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
     const int32_t* idx = p.idx + (int64_t)b * p.top_k;
     const int64_t tok_stride = (int64_t)p.HG * D;
 
-    // list positions -> token positions of the rows of iteration `it` that this lane group loads
-    auto lookup = [&](int it, int (&pos)[DEC_UN]) {
+    // list positions -> token positions of the rows of iteration `it` that this lane copies
+    auto lookup = [&](int it, int (&pos)[PER_LANE]) {
 #pragma unroll
-        for (int u = 0; u < DEC_UN; ++u) {
-            const int j = it * KEYS_PER_ITER + u * GROUPS + gi;
+        for (int i = 0; i < PER_LANE; ++i) {
+            const int j = it * DEC_ROWS + my_row + i * ROWS_PER_PASS;
             int q = -1;
             if (it < it_end && j < n_att) {
                 if (j < i_end) q = j;
                 else if (j < n_glob) q = __ldg(idx + (j - i_end));
                 else q = m_end + (j - n_glob);
             }
-            pos[u] = q;
+            pos[i] = q;
         }
     };
-    auto issue = [&](int stage, const int (&pos)[DEC_UN]) {
-        uint8_t* sk = ring + stage * STAGE_BYTES;
-        uint8_t* sv = sk + KEYS_PER_ITER * D * 2;
+    auto issue = [&](int stage, const int (&pos)[PER_LANE]) {
+        uint4* sk = ring + stage * STAGE_CHUNKS;
+        uint4* sv = sk + TILE_CHUNKS;
 #pragma unroll
-        for (int u = 0; u < DEC_UN; ++u) {
-            const int64_t off = (int64_t)(pos[u] < 0 ? 0 : pos[u]) * tok_stride;
-            const int o = ((u * GROUPS + gi) * LPR + li) * 16;
-            cp_async16(sk + o, Kb + off, pos[u] < 0 ? 0 : 16);
-            cp_async16(sv + o, Vb + off, pos[u] < 0 ? 0 : 16);
+        for (int i = 0; i < PER_LANE; ++i) {
+            const int r = my_row + i * ROWS_PER_PASS;
+            const int64_t off = (int64_t)(pos[i] < 0 ? 0 : pos[i]) * tok_stride;
+            cp_async16(&sk[swz<CH>(r, my_chunk)], Kb + off, pos[i] < 0 ? 0 : 16);
+            cp_async16(&sv[swz<CH>(r, my_chunk)], Vb + off, pos[i] < 0 ? 0 : 16);
         }
     };
 
-    // this lane's 8 columns of the G query rows, pre-scaled into the exp2 domain
-    float q[G][8];
+    // B fragments of Q^T for every 16-wide slice of D: element (k = d, n = head); heads >= G are zero
+    uint32_t qb[D / 16][2];
+    {
+        const int head = lane >> 2;
+        const __nv_bfloat16* qrow = p.Q + ((int64_t)b * p.H + kvh * G + (head < G ? head : 0)) * D;
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p.Q + ((int64_t)b * p.H + kvh * G + g) * D + li * 8);
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float2 f = __bfloat1622float2(h[i]);
-            q[g][2 * i] = f.x * p.scale_log2;
-            q[g][2 * i + 1] = f.y * p.scale_log2;
+        for (int ks = 0; ks < D / 16; ++ks) {
+            const int d0 = ks * 16 + 2 * (lane & 3);
+            qb[ks][0] = head < G ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
+            qb[ks][1] = head < G ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
         }
     }
-    float m[G], l[G], acc[G][8];
+    // this thread's two heads (columns 2 (lane & 3), +1): running maximum and its share of the sum;
+    // O^T: D / 16 tiles of (16 values of d) x (8 heads), c-fragment layout
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float o_acc[D / 16][4];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        m[g] = -INFINITY;
-        l[g] = 0.f;
+    for (int i = 0; i < D / 16; ++i)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
-    }
+        for (int j = 0; j < 4; ++j) o_acc[i][j] = 0.f;
 
     // prologue: DEC_STAGES - 1 iterations in flight, positions of one more in registers
-    int pos_next[DEC_UN];
+    int pos_next[PER_LANE];
     const int it0 = it_begin + warp;
 #pragma unroll
     for (int s = 0; s < DEC_STAGES - 1; ++s) {
@@ -424,107 +425,92 @@ attend_decode_kernel(AttendParams p) {
         lookup(it + DEC_STAGES * DEC_WARPS, pos_next);
         cp_async_wait<DEC_STAGES - 1>();
         __syncwarp();
-        const uint8_t* sk = ring + (n % DEC_STAGES) * STAGE_BYTES;
-        const uint8_t* sv = sk + KEYS_PER_ITER * D * 2;
-        bool ok[DEC_UN];
-        float sc[DEC_UN][G];
+        const uint4* tk = ring + (n % DEC_STAGES) * STAGE_CHUNKS;
+        const uint4* tv = tk + TILE_CHUNKS;
+
+        // S^T[key, head] = K Q^T
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int u = 0; u < DEC_UN; ++u) {
-            ok[u] = it * KEYS_PER_ITER + u * GROUPS + gi < n_att;
-            const uint4 kr = *reinterpret_cast<const uint4*>(sk + ((u * GROUPS + gi) * LPR + li) * 16);
-            float kf[8];
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&kr);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 f = __bfloat1622float2(h[i]);
-                kf[2 * i] = f.x;
-                kf[2 * i + 1] = f.y;
-            }
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float a = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) a = fmaf(q[g][i], kf[i], a);
-                sc[u][g] = a;
-            }
+        for (int ks = 0; ks < D / 16; ++ks) {
+            uint32_t a[4];
+            load_a_frag<CH>(a, tk, 0, ks * 2, lane);
+            mma_bf16_16816(sc, a, qb[ks][0], qb[ks][1]);
         }
+        // rows lane / 4 and + 8 of the tile; list positions past the end are masked
+        const int key_lo = it * DEC_ROWS + (lane >> 2);
+        const bool ok_lo = key_lo < n_att, ok_hi = key_lo + 8 < n_att;
+        sc[0] = ok_lo ? sc[0] * p.scale_log2 : -INFINITY;
+        sc[1] = ok_lo ? sc[1] * p.scale_log2 : -INFINITY;
+        sc[2] = ok_hi ? sc[2] * p.scale_log2 : -INFINITY;
+        sc[3] = ok_hi ? sc[3] * p.scale_log2 : -INFINITY;
+        float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
 #pragma unroll
-        for (int o = LPR / 2; o >= 1; o >>= 1)
-#pragma unroll
-            for (int u = 0; u < DEC_UN; ++u)
-#pragma unroll
-                for (int g = 0; g < G; ++g) sc[u][g] += __shfl_xor_sync(0xffffffffu, sc[u][g], o);
-        // online softmax per head, then the value rows
-        float vf[DEC_UN][8];
-#pragma unroll
-        for (int u = 0; u < DEC_UN; ++u) {
-            const uint4 vr = *reinterpret_cast<const uint4*>(sv + ((u * GROUPS + gi) * LPR + li) * 16);
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&vr);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 f = __bfloat1622float2(h[i]);
-                vf[u][2 * i] = f.x;
-                vf[u][2 * i + 1] = f.y;
-            }
+        for (int o = 4; o < 32; o <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
         }
+        const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        if (mn0 != m_run[0] || mn1 != m_run[1]) {          // uniform over the lanes that share the heads
+            const float al0 = fast_exp2(m_run[0] - ms0), al1 = fast_exp2(m_run[1] - ms1);
+            l_run[0] *= al0;
+            l_run[1] *= al1;
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float mx = -INFINITY;
-#pragma unroll
-            for (int u = 0; u < DEC_UN; ++u) mx = fmaxf(mx, ok[u] ? sc[u][g] : -INFINITY);
-            const float m_new = fmaxf(m[g], mx);
-            const float ms = (m_new == -INFINITY) ? 0.f : m_new;
-            const float alpha = fast_exp2(m[g] - ms);
-            m[g] = m_new;
-            float pw[DEC_UN], sum = 0.f;
-#pragma unroll
-            for (int u = 0; u < DEC_UN; ++u) {
-                pw[u] = ok[u] ? fast_exp2(sc[u][g] - ms) : 0.f;
-                sum += pw[u];
+            for (int i = 0; i < D / 16; ++i) {
+                o_acc[i][0] *= al0; o_acc[i][1] *= al1; o_acc[i][2] *= al0; o_acc[i][3] *= al1;
             }
-            l[g] = l[g] * alpha + sum;
+            m_run[0] = mn0;
+            m_run[1] = mn1;
+        }
+        const float p0 = fast_exp2(sc[0] - ms0), p1 = fast_exp2(sc[1] - ms1);
+        const float p2 = fast_exp2(sc[2] - ms0), p3 = fast_exp2(sc[3] - ms1);
+        l_run[0] += p0 + p2;
+        l_run[1] += p1 + p3;
+        // P^T as the B operand (k = key, n = head): thread T needs keys 2 (T & 3), +1 (and + 8) of head T / 4;
+        // in the accumulator layout those sit in lanes (key & 7) * 4 + head / 2, packed per head pair.
+        const uint32_t w_lo = pack_bf16(p0, p1), w_hi = pack_bf16(p2, p3);       // keys r and r + 8, heads 2q, 2q + 1
+        const int src0 = (2 * (lane & 3)) * 4 + (lane >> 3), src1 = src0 + 4;
+        const uint32_t a_lo = __shfl_sync(0xffffffffu, w_lo, src0), b_lo = __shfl_sync(0xffffffffu, w_lo, src1);
+        const uint32_t a_hi = __shfl_sync(0xffffffffu, w_hi, src0), b_hi = __shfl_sync(0xffffffffu, w_hi, src1);
+        const uint32_t sel = ((lane >> 2) & 1) ? 0x7632u : 0x5410u;               // odd head: upper halves, else lower
+        const uint32_t pb0 = __byte_perm(a_lo, b_lo, sel), pb1 = __byte_perm(a_hi, b_hi, sel);
+        // O^T[d, head] += V^T P^T: A = V^T from the row-major V tile through transposing ldmatrix
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float a = acc[g][i] * alpha;
-#pragma unroll
-                for (int u = 0; u < DEC_UN; ++u) a = fmaf(pw[u], vf[u][i], a);
-                acc[g][i] = a;
-            }
+        for (int dt = 0; dt < D / 16; ++dt) {
+            uint32_t av[4];
+            const int r = (lane & 7) + ((lane >> 4) & 1) * 8;          // key row of this lane's matrix
+            const int c = dt * 2 + ((lane >> 3) & 1);                 // 16-byte chunk: d 0-7 or 8-15 of the tile
+            ldmatrix_x4_trans(av, tv + swz<CH>(r, c));
+            mma_bf16_16816(o_acc[dt], av, pb0, pb1);
         }
         __syncwarp();          // the stage is free for the copy issued next iteration
     }
     cp_async_wait<0>();
 
-    // merge the lane groups of the warp (same columns li, different rows)
+    // the lanes that share a head pair (same lane & 3) each saw different rows: add their sums
 #pragma unroll
-    for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            const float m_o = __shfl_xor_sync(0xffffffffu, m[g], o);
-            const float l_o = __shfl_xor_sync(0xffffffffu, l[g], o);
-            const float m_new = fmaxf(m[g], m_o);
-            const float ms = (m_new == -INFINITY) ? 0.f : m_new;
-            const float a = fast_exp2(m[g] - ms), bsc = fast_exp2(m_o - ms);
-            l[g] = l[g] * a + l_o * bsc;
-            m[g] = m_new;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float v_o = __shfl_xor_sync(0xffffffffu, acc[g][i], o);
-                acc[g][i] = acc[g][i] * a + v_o * bsc;
-            }
-        }
+    for (int o = 4; o < 32; o <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
     }
     // merge the warps through shared memory (the rings are idle now)
     __syncthreads();
-    float* s_m = reinterpret_cast<float*>(dec_smem);          // [DEC_WARPS][G]
-    float* s_l = s_m + DEC_WARPS * G;                          // [DEC_WARPS][G]
-    float* s_acc = s_l + DEC_WARPS * G;                        // [DEC_WARPS][G][D]
-    if (gi == 0) {
+    float* s_m = reinterpret_cast<float*>(dec_smem);          // [DEC_WARPS][8]
+    float* s_l = s_m + DEC_WARPS * 8;                          // [DEC_WARPS][8]
+    float* s_acc = s_l + DEC_WARPS * 8;                        // [DEC_WARPS][8][D]
+    {
+        const int h0 = 2 * (lane & 3);
+        if (lane < 4) {
+            s_m[warp * 8 + h0] = m_run[0]; s_m[warp * 8 + h0 + 1] = m_run[1];
+            s_l[warp * 8 + h0] = l_run[0]; s_l[warp * 8 + h0 + 1] = l_run[1];
+        }
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            if (li == 0) { s_m[warp * G + g] = m[g]; s_l[warp * G + g] = l[g]; }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) s_acc[(warp * G + g) * D + li * 8 + i] = acc[g][i];
+        for (int dt = 0; dt < D / 16; ++dt) {
+            const int d0 = dt * 16 + (lane >> 2);
+            s_acc[(warp * 8 + h0) * D + d0] = o_acc[dt][0];
+            s_acc[(warp * 8 + h0 + 1) * D + d0] = o_acc[dt][1];
+            s_acc[(warp * 8 + h0) * D + d0 + 8] = o_acc[dt][2];
+            s_acc[(warp * 8 + h0 + 1) * D + d0 + 8] = o_acc[dt][3];
         }
     }
     __syncthreads();
@@ -533,14 +519,14 @@ attend_decode_kernel(AttendParams p) {
         const int g = e / D, col = e % D;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, s_m[w * G + g]);
+        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, s_m[w * 8 + g]);
         const float Ms = (M == -INFINITY) ? 0.f : M;
         float o = 0.f, lsum = 0.f;
 #pragma unroll
         for (int w = 0; w < DEC_WARPS; ++w) {
-            const float wgt = fast_exp2(s_m[w * G + g] - Ms);
-            o += wgt * s_acc[(w * G + g) * D + col];
-            lsum += wgt * s_l[w * G + g];
+            const float wgt = fast_exp2(s_m[w * 8 + g] - Ms);
+            o += wgt * s_acc[(w * 8 + g) * D + col];
+            lsum += wgt * s_l[w * 8 + g];
         }
         if (p.nsplit == 1) {
             p.O[((int64_t)b * p.H + kvh * G + g) * D + col] = __float2bfloat16_rn(o / lsum);
@@ -554,15 +540,14 @@ attend_decode_kernel(AttendParams p) {
 
 template <int D, int G>
 static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
-    constexpr int keys_per_iter = (32 / (D / 8)) * DEC_UN;
-    constexpr int smem = DEC_WARPS * DEC_STAGES * 2 * keys_per_iter * D * 2;
-    static_assert(smem >= (2 * DEC_WARPS * G + DEC_WARPS * G * D) * 4, "the warp merge reuses the rings");
+    constexpr int smem = DEC_WARPS * DEC_STAGES * 2 * DEC_ROWS * D * 2;
+    static_assert(smem >= (2 * DEC_WARPS * 8 + DEC_WARPS * 8 * D) * 4, "the warp merge reuses the rings");
     cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int per_sm = 1;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_decode_kernel<D, G>, DEC_WARPS * 32, smem);
     if (e != cudaSuccess) return e;
-    const int iters = (n_att_max + keys_per_iter - 1) / keys_per_iter;
+    const int iters = (n_att_max + DEC_ROWS - 1) / DEC_ROWS;
     // one wave of CTAs, each warp with at least a few iterations
     int nsplit = (per_sm * ctx->num_sms) / (p.HG * B);
     if (nsplit > kAttMaxSplits) nsplit = kAttMaxSplits;
