@@ -319,8 +319,8 @@ def time_decode(cfg3, n_steps, rank_seed):
     K = torch.randn(B, n, cfg3.H_G, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
     V = torch.randn(B, n, cfg3.H_G, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
     Qs = torch.randn(n_steps, B, 1, cfg3.H, cfg3.d, device="cuda", dtype=torch.bfloat16, generator=g)
-    Knew = K[:, S:].clone()
-    Vnew = V[:, S:].clone()
+    Knew = K[:, S:].transpose(0, 1).contiguous().unsqueeze(2)      # [step, B, 1, H_G, d]: one contiguous block per step
+    Vnew = V[:, S:].transpose(0, 1).contiguous().unsqueeze(2)
     Kc = torch.zeros(B, n, cfg3.d_c, dtype=torch.bfloat16, device="cuda")
     for r0 in range(0, S, 4096):
         ctx.compress_keys(K[:, r0: r0 + 4096].contiguous(), Kc, [r0] * B)
@@ -330,9 +330,9 @@ def time_decode(cfg3, n_steps, rank_seed):
 
     def step(i):
         t = [S + i] * B
-        kn, vn = Knew[:, i: i + 1], Vnew[:, i: i + 1]
-        ctx.append_kv(kn.contiguous(), vn.contiguous(), K, V, t)
-        ctx.compress_keys(kn.contiguous(), Kc, t)
+        kn, vn = Knew[i], Vnew[i]
+        ctx.append_kv(kn, vn, K, V, t)
+        ctx.compress_keys(kn, Kc, t)
         ctx.select(Qs[i], Kc, t, idx, n_sel)
         ctx.attend(Qs[i], K, V, t, idx, n_sel, O)
 

@@ -115,26 +115,27 @@ def load_library():
 
 
 def _ptr(t: Optional[torch.Tensor]):
-    return C.c_void_p(0 if t is None else t.data_ptr())
+    return 0 if t is None else t.data_ptr()
 
 
 def _check(t: torch.Tensor, name: str, dtype, shape=None):
-    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+    # kept cheap: it runs for every tensor of every call
+    if not t.is_cuda:
         raise TypeError(f"{name} must be a CUDA tensor")
     if t.dtype != dtype:
         raise TypeError(f"{name} must have dtype {dtype}, got {t.dtype}")
     if not t.is_contiguous():
         raise ValueError(f"{name} must be contiguous")
-    if shape is not None and tuple(t.shape) != tuple(shape):
+    if shape is not None and t.shape != shape:
         raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
 
 
-def _stream_ptr(stream) -> C.c_void_p:
+def _stream_ptr(stream) -> int:
     if stream is None:
-        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        return torch.cuda.current_stream().cuda_stream
     if isinstance(stream, int):
-        return C.c_void_p(stream)
-    return C.c_void_p(stream.cuda_stream)
+        return stream
+    return stream.cuda_stream
 
 
 class Esa:
@@ -194,10 +195,10 @@ class Esa:
 
     @staticmethod
     def _nprev(n_prev: Sequence[int], B: int):
-        a = np.ascontiguousarray(np.asarray(n_prev, dtype=np.int64).reshape(-1))
-        if a.shape[0] != B:
+        """Host int64[B] for the C call (a ctypes array: cheaper to build than a numpy one)."""
+        if len(n_prev) != B:
             raise ValueError("n_prev must have one entry per sequence")
-        return a
+        return (C.c_int64 * B)(*[int(x) for x in n_prev])
 
     # ------------------------------------------------------------ entry points
     def append_kv(self, K_new, V_new, K_cache, V_cache, n_prev, stream=None, sync=False):
@@ -210,10 +211,10 @@ class Esa:
         npv = self._nprev(n_prev, B)
         if sync:
             st = self.lib.esa_append_kv(self._h, B, _ptr(K_new), _ptr(V_new), n_new, _ptr(K_cache),
-                                        _ptr(V_cache), npv.ctypes.data_as(C.c_void_p))
+                                        _ptr(V_cache), npv)
         else:
             st = self.lib.esa_append_kv_async(self._h, B, _ptr(K_new), _ptr(V_new), n_new, _ptr(K_cache),
-                                              _ptr(V_cache), npv.ctypes.data_as(C.c_void_p),
+                                              _ptr(V_cache), npv,
                                               _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_append_kv")
@@ -226,10 +227,10 @@ class Esa:
         npv = self._nprev(n_prev, B)
         if sync:
             st = self.lib.esa_compress_keys(self._h, B, _ptr(K_new), n_new, _ptr(kc_cache),
-                                            npv.ctypes.data_as(C.c_void_p))
+                                            npv)
         else:
             st = self.lib.esa_compress_keys_async(self._h, B, _ptr(K_new), n_new, _ptr(kc_cache),
-                                                  npv.ctypes.data_as(C.c_void_p), _stream_ptr(stream))
+                                                  npv, _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_compress_keys")
 
@@ -243,10 +244,10 @@ class Esa:
         npv = self._nprev(n_prev, B)
         if sync:
             st = self.lib.esa_select(self._h, B, _ptr(Q_cur), l_C, _ptr(kc_cache),
-                                     npv.ctypes.data_as(C.c_void_p), _ptr(idx_out), _ptr(n_sel_out))
+                                     npv, _ptr(idx_out), _ptr(n_sel_out))
         else:
             st = self.lib.esa_select_async(self._h, B, _ptr(Q_cur), l_C, _ptr(kc_cache),
-                                           npv.ctypes.data_as(C.c_void_p), _ptr(idx_out), _ptr(n_sel_out),
+                                           npv, _ptr(idx_out), _ptr(n_sel_out),
                                            _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_select")
@@ -263,10 +264,10 @@ class Esa:
         npv = self._nprev(n_prev, B)
         if sync:
             st = self.lib.esa_attend(self._h, B, _ptr(Q_cur), l_C, _ptr(K_cache), _ptr(V_cache),
-                                     npv.ctypes.data_as(C.c_void_p), _ptr(idx), _ptr(n_sel), _ptr(O))
+                                     npv, _ptr(idx), _ptr(n_sel), _ptr(O))
         else:
             st = self.lib.esa_attend_async(self._h, B, _ptr(Q_cur), l_C, _ptr(K_cache), _ptr(V_cache),
-                                           npv.ctypes.data_as(C.c_void_p), _ptr(idx), _ptr(n_sel), _ptr(O),
+                                           npv, _ptr(idx), _ptr(n_sel), _ptr(O),
                                            _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_attend")
@@ -295,6 +296,6 @@ def attend_noalloc(cfg: EsaConfig, Q_cur, K_cache, V_cache, n_prev, idx, n_sel, 
     npv = Esa._nprev(n_prev, B)
     c = cfg.to_c()
     st = lib.esa_attend_noalloc(C.byref(c), B, _ptr(Q_cur), l_C, _ptr(K_cache), _ptr(V_cache),
-                                npv.ctypes.data_as(C.c_void_p), _ptr(idx), _ptr(n_sel), _ptr(O), _stream_ptr(stream))
+                                npv, _ptr(idx), _ptr(n_sel), _ptr(O), _stream_ptr(stream))
     if st != 0:
         raise EsaError(st, "esa_attend_noalloc")
