@@ -13,9 +13,13 @@
 // Rows of the MMA tile are (query, head-in-group) pairs, row = c * G + g with
 // G = H / H_G, so one K/V tile gathered for a key/value head serves all G query heads
 // that share it.  Flash-style online softmax in the exp2 domain, bf16 operands, fp32
-// scores and accumulators.  Small chunks (decode) split the key list across CTAs and a
-// second kernel merges the partial (O, m, l) triples -- the same algebra as Algorithm 1's
-// merge.
+// scores and accumulators.
+//
+// This file holds the kernels for small chunks: a generic split-KV mma.sync kernel
+// (up to 64 rows per key/value head), the streaming kernel for decode (one query per
+// sequence), the kernel that merges the partial (O, m, l) triples of key-list splits -- the
+// same algebra as Algorithm 1's merge -- and the entry point that needs no allocation.
+// Prefill-sized chunks run in esa_attend_tc.cu.
 #include "esa_internal.h"
 
 namespace esa {

@@ -6,7 +6,7 @@
 // Ties are the rule, not the exception (each query's arg-max scores exactly 0 and the
 // pooling copies every peak to 2*eps+1 neighbours), so the order is total: larger score
 // first, lower index first among equal scores.  Scores are handled as order-preserving
-// uint32 keys.  One thread-block cluster works on one sequence: every CTA pools its
+// uint32 keys.  One thread-block cluster (8 CTAs, or 16 for small batches) works on one sequence: every CTA pools its
 // slice of M, then three radix passes (11 + 11 + 10 bits, each digit's histogram all-reduced
 // into every CTA through distributed shared memory) find the k-th largest key T, and an index-ordered
 // compaction emits every key > T plus the first (k - #greater) keys == T, which is
