@@ -269,6 +269,33 @@ def test_c3_decode_steps():
                 hp.check_attention(O[b], res.O, what=f"c3 step {step} seq {b}")
 
 
+# ------------------------------------------- batch of ragged sequences, d' = 64
+def test_batch_of_ragged_sequences_dc64():
+    """Two sequences at different positions in one call (different partitions, one with every middle
+    token selected and one scored), compressed dimension 64: the tensor-core kernels' other
+    instantiation and the per-sequence bookkeeping."""
+    cfg = syn.get_config("c2").with_(H=8, H_G=2, d_c=64, l_C=256, l_I=16, l_L=512, k=512, S=6144, B=2)
+    p = hp.oracle_params(cfg)
+    _, _, Wq, Wk = hp.oracle_weights(cfg)
+    l_C = cfg.l_C
+    t_list = [768, 5000]                       # |M| = 240 (all selected) and 4472 (scored)
+    n = max(t_list) + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=2)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, B=2)
+    seq.fill_kv(0, n)
+    fill_kc_gpu(ctx, seq, n, step=1024)
+    Q = torch.stack([hp.bits_to_torch(syn.qkv_rows(cfg, "q", t, t + l_C, 0, b)) for b, t in enumerate(t_list)]).contiguous()
+    sel, O = run_step_gpu(ctx, seq, Q, t_list, do_compress=False)
+    for b, t in enumerate(t_list):
+        K64 = hp.torch_to_f64(seq.K[b, : t + l_C])
+        V64 = hp.torch_to_f64(seq.V[b, : t + l_C])
+        res = orc.esa_step(hp.torch_to_f64(Q[b]), K64, V64, Wq, Wk, p, t)
+        nd = hp.check_index_sets(sel[b], res, cfg.k, what=f"ragged seq {b}")
+        if nd == 0:
+            hp.check_attention(O[b], res.O, what=f"ragged seq {b}")
+        hp.check_compressed(seq.Kc[b, : t], K64[:t].reshape(t, -1), Wk, what=f"ragged seq {b} cache")
+
+
 # ----------------------------------------------------------------- error paths
 def test_argument_errors_leave_outputs_untouched():
     import paper_2502_14477_b200 as esa
