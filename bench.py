@@ -38,6 +38,10 @@ import torch
 import esa_synth as syn
 
 N_LAYERS_STACK = 32
+# dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised in
+# profiles/dram_bytes_per_kernel.txt (same kernels, same launch shapes as the timed workloads).
+ATTEND_TC_DRAM_BYTES = 32504832 + 471296
+DECODE_STEP_DRAM_BYTES = (205785856 + 1053440) + 541184 + 39168 + 303104 + 1134848 + (264000256 + 3063552) + 4179456
 
 
 # ----------------------------------------------------------------------------
@@ -410,7 +414,8 @@ def run_esa(args, cfg):
     att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
     achieved = att_flops / (att_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (+ attend_merge_kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": ATTEND_TC_DRAM_BYTES,
+                "traffic_unit": "bytes per attend_tc_kernel launch (ncu, profiles/dram_bytes_per_kernel.txt)",
                 "peak_source": peaks["source"] + " sustained bf16", "share_of_step": att_ms / (ms_total),
                 "launches": len(events)}
 
@@ -453,7 +458,8 @@ def run_esa(args, cfg):
         decode = {"workload": "c3: 8 sequences x 131072 cached tokens, 1 query each, k=4096 l_L=2048 l_I=128",
                   "us_per_step": us, "steps": args.decode_steps, "launches_per_step": lps,
                   "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                               "frac": gbs / peaks["hbm_gbs"], "traffic": DECODE_STEP_DRAM_BYTES,
+                               "traffic_unit": "bytes per decode step, all kernels (ncu, profiles/dram_bytes_per_kernel.txt)",
                                "algorithmic_bytes_per_step": byts, "peak_source": peaks["source"] + " copy"}}
 
     if rank != 0:
