@@ -29,8 +29,8 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, att, status, total;
-    size_t att_elems;
+    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, att, att_count, status, total;
+    size_t att_elems, att_count_elems;
 };
 
 Layout make_layout(const esa_config* c) {
@@ -51,9 +51,11 @@ Layout make_layout(const esa_config* c) {
     if (rows > (size_t)kAttSplitRows) rows = kAttSplitRows;
     L.att_elems = (size_t)c->max_batch * c->n_kv_heads * kAttMaxSplits * rows * (c->head_dim + 2);
     // prefill-sized chunks: room for one sequence's key list split kAttPrefillSplits ways
-    const size_t big = (size_t)c->n_kv_heads * kAttPrefillSplits * c->max_chunk * G * (c->head_dim + 2);
+    const size_t big = (size_t)c->n_kv_heads * kAttPrefillSplits * (c->max_chunk * G + 1) * (c->head_dim + 2);
     if ((size_t)c->max_chunk * G > (size_t)kAttSplitRows && big > L.att_elems) L.att_elems = big;
     L.att = take(4 * L.att_elems);
+    L.att_count_elems = (size_t)c->max_batch * c->n_kv_heads * ((c->max_chunk * G + 255) / 256);
+    L.att_count = take(4 * L.att_count_elems);
     L.status = take(256);
     L.total = off;
     return L;
@@ -159,8 +161,11 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
     c->att_part = reinterpret_cast<float*>(base + L.att);
     c->att_part_elems = L.att_elems;
+    c->att_count = reinterpret_cast<int*>(base + L.att_count);
+    c->att_count_elems = L.att_count_elems;
     c->status = reinterpret_cast<int*>(base + L.status);
-    if (cudaMemset(c->status, 0, 256) != cudaSuccess) {
+    if (cudaMemset(c->status, 0, 256) != cudaSuccess ||
+        cudaMemset(c->att_count, 0, 4 * L.att_count_elems) != cudaSuccess) {
         cudaFree(base);
         delete c;
         return ESA_ERR_CUDA;

@@ -630,17 +630,9 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
     }
     const int R = l_C * ctx->G;
     if (R > kAttSplitRows) {
-        // prefill-sized chunks: tcgen05 kernel, then the merge when it split the key list
+        // prefill-sized chunks: tcgen05 kernel (a split key list is merged inside it)
         int nsplit = 1;
-        cudaError_t e = launch_attend_tc(ctx, B, l_C, Q, K, V, meta, idx, n_sel, O, n_att_max, st, &nsplit);
-        if (e != cudaSuccess) return e;
-        if (nsplit > 1) {
-            p.nsplit = nsplit;
-            if (ctx->d == 128) e = launch_pdl(attend_merge_kernel<128>, dim3((R + 7) / 8, p.HG, B), dim3(256), 0, st, p);
-            else e = launch_pdl(attend_merge_kernel<64>, dim3((R + 7) / 8, p.HG, B), dim3(256), 0, st, p);
-            ctx->launches += 1;
-        }
-        return e;
+        return launch_attend_tc(ctx, B, l_C, Q, K, V, meta, idx, n_sel, O, n_att_max, st, &nsplit);
     }
     if (l_C == 1) {
         // decode: streaming kernel for the usual group sizes

@@ -29,7 +29,8 @@
 //     rescaling O in tensor memory rare; (O, m, l) stay consistent, so the final division,
 //     or the split merge, needs no correction.
 //   * A long key list can be split across CTAs (blockIdx.z); partial (O, m, l) go to the
-//     context's scratch and the merge kernel of esa_attend.cu combines them.
+//     context's scratch through coalesced stores, and the CTA that finishes a unit last merges
+//     them with its own accumulator (an arrival counter per unit decides; nobody waits).
 #include <cstring>
 
 #include "esa_internal.h"
@@ -53,6 +54,7 @@ constexpr int TC_PRODUCERS = TC_PRODUCER_WARPS * 32;
 constexpr int TC_REGS_LAUNCH = 128;
 constexpr int TC_REGS_SOFTMAX = 168;
 constexpr int TC_REGS_OTHER = 88;
+static_assert(kAttPrefillSplits == 4, "the in-kernel merge selects among four weights");
 static_assert(8 * TC_REGS_SOFTMAX + 8 * TC_REGS_OTHER <= 16 * TC_REGS_LAUNCH,
               "register split exceeds the CTA's launch allocation: setmaxnreg.inc would never return");
 constexpr int TC_POLY_PAIRS_OF_4 = 1; // of every 4 column pairs, this many take 2^x on the FMA pipe
@@ -70,6 +72,8 @@ struct TcAttendParams {
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
+    int Rp;             // rows of a scratch part (R rounded up to even: 16-byte aligned parts)
+    int* unit_count;    // arrivals per (sequence, key/value head, row tile); returns to 0 after each launch
     int q_tma;          // Q tiles arrive by TMA (one arrival) instead of cp.async (one per producer thread)
     float scale_log2;
     SeqMeta meta;
@@ -159,6 +163,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int merge_ticket;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int warp_u = __shfl_sync(0xffffffffu, warp, 0);     // provably warp-uniform copy
@@ -334,24 +339,148 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 }
             }
         } else {
-            float* dst = p.part + ((((int64_t)b * p.HG + kvh) * p.nsplit + split) * R + (row_ok ? row : 0)) * (D + 2);
+            // ---- split key list.  Every CTA leaves its partial (O, m, l) in the scratch; the CTA that
+            // finishes a (sequence, head, row tile) unit last combines the others' partials with its own,
+            // which is still in tensor memory, and writes the rows of O: no CTA waits for another one.
+            // Scratch of part s: O rows [Rp][D] fp32, then (m, l) pairs [Rp][2].
+            constexpr int DH = D / 2;                  // columns handled per round
+            constexpr int NC = DH / 4;                 // float4 per staged row: 16 or 8
+            const int Rp = p.Rp;
+            float* unit_base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit) * (int64_t)Rp * (D + 2);
+            const int64_t part_stride = (int64_t)Rp * (D + 2);
+            float* myO = unit_base + split * part_stride;
+            // Staging for coalesced traffic: this warp's quarter of its own Q tile, 32 rows x DH fp32.
+            // Free by now: O_READY covers every Q K^T of the tile.  16-byte cells are XOR-swizzled by
+            // the row so that row-per-lane and row-per-half-warp accesses are both conflict-free.
+            float4* stage = reinterpret_cast<float4*>(sQ + qt * Q_TILE_BYTES + (warp_u & 3) * (Q_TILE_BYTES / 4));
+            const int wrow0 = row0 + qt * 128 + lane_base;        // first row of this warp
             if (n_tiles > 0) {
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c0, o);
-                    tmem_wait_ld();
-                    if (row_ok) {
+                    for (int cc = 0; cc < DH; cc += 32) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + h * DH + cc, o);
+                        tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2)
-                            *reinterpret_cast<float2*>(dst + c0 + i) =
-                                make_float2(__uint_as_float(o[i]), __uint_as_float(o[i + 1]));
+                        for (int q4 = 0; q4 < 8; ++q4)
+                            stage[lane * NC + ((cc / 4 + q4) ^ (lane & (NC - 1)))] =
+                                make_float4(__uint_as_float(o[4 * q4]), __uint_as_float(o[4 * q4 + 1]),
+                                            __uint_as_float(o[4 * q4 + 2]), __uint_as_float(o[4 * q4 + 3]));
                     }
+                    __syncwarp();
+#pragma unroll 4
+                    for (int it = 0; it < NC; ++it) {
+                        const int e = it * 32 + lane, rr = e / NC, c = e % NC;
+                        const float4 val = stage[rr * NC + (c ^ (rr & (NC - 1)))];
+                        if (wrow0 + rr < R)
+                            __stcg(reinterpret_cast<float4*>(myO + (int64_t)(wrow0 + rr) * D + h * DH) + c, val);
+                    }
+                    __syncwarp();
                 }
             }
-            if (row_ok) {
-                dst[D] = m_run;        // -inf marks an empty part
-                dst[D + 1] = l_run;
+            if (row_ok) __stcg(reinterpret_cast<float2*>(myO + (int64_t)Rp * D) + row, make_float2(m_run, l_run));   // m = -inf: empty part
+            __threadfence();
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            if (tid == 0) {
+                int* cnt = p.unit_count + ((int64_t)b * p.HG + kvh) * gridDim.x + blockIdx.x;
+                const int ticket = atomicAdd(cnt, 1);
+                if (ticket == p.nsplit - 1) *cnt = 0;          // ready for the next launch
+                merge_ticket = ticket;
+            }
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            if (merge_ticket == p.nsplit - 1) {
+                __threadfence();
+                // weights of the parts in the log2 domain (Algorithm 1's merge of (O, m, l))
+                float w[kAttPrefillSplits];
+                float m_max = m_run;
+                float2 ml[kAttPrefillSplits];
+#pragma unroll
+                for (int s = 0; s < kAttPrefillSplits; ++s) {
+                    ml[s] = make_float2(-INFINITY, 0.f);
+                    if (s < p.nsplit && s != split && row_ok)
+                        ml[s] = __ldcg(reinterpret_cast<const float2*>(unit_base + s * part_stride + (int64_t)Rp * D) + row);
+                    if (s == split) ml[s] = make_float2(m_run, l_run);
+                    m_max = fmaxf(m_max, ml[s].x);
+                }
+                float den = 0.f;
+#pragma unroll
+                for (int s = 0; s < kAttPrefillSplits; ++s) {
+                    w[s] = (ml[s].x == -INFINITY) ? 0.f : fast_exp2(ml[s].x - m_max);
+                    den += w[s] * ml[s].y;
+                }
+                const float inv = 1.f / den;
+                auto pick = [&](int s) { return s == 0 ? w[0] : s == 1 ? w[1] : s == 2 ? w[2] : w[3]; };   // no dynamic register indexing
+                __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;
+                // The other parts' rows arrive through a ring of two shared-memory buffers per warp
+                // (16-byte cp.async, all copies of a buffer in flight together), in the order
+                // (column half, part).  The K/V stages serve as the ring: both warpgroups have passed
+                // their O_READY before the arrival barrier above, so no MMA reads them any more.
+                float4* ring = reinterpret_cast<float4*>(sK + warp_u * (2 * TC_STAGES * KV_TILE_BYTES / 8));
+                const int n_other = p.nsplit - 1, n_pairs = 2 * n_other;
+                auto other = [&](int i) { const int s = i % n_other; return s + (s >= split ? 1 : 0); };
+                auto issue = [&](int i) {
+                    const int h = i / n_other;
+                    const float* srcO = unit_base + other(i) * part_stride + h * DH;
+                    float4* buf = ring + (i & 1) * (32 * NC);
+#pragma unroll
+                    for (int it = 0; it < NC; ++it) {
+                        const int e = it * 32 + lane, rr = e / NC, c = e % NC;
+                        const bool ok = wrow0 + rr < R;
+                        cp_async16(buf + rr * NC + (c ^ (rr & (NC - 1))), srcO + (int64_t)(ok ? wrow0 + rr : 0) * D + c * 4,
+                                   ok ? 16 : 0);
+                    }
+                    cp_async_commit();
+                };
+                issue(0);
+                if (n_pairs > 1) issue(1);
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    float acc[DH];
+                    {
+                        const float wo = pick(split) * inv;       // 0 when this CTA's own part is empty
+#pragma unroll
+                        for (int cc = 0; cc < DH; cc += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + h * DH + cc, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[cc + i] = (wo == 0.f) ? 0.f : __uint_as_float(o[i]) * wo;
+                        }
+                    }
+#pragma unroll 1
+                    for (int k = 0; k < n_other; ++k) {
+                        const int i = h * n_other + k;
+                        if (i + 1 < n_pairs) cp_async_wait<1>();
+                        else cp_async_wait<0>();
+                        __syncwarp();
+                        const float4* buf = ring + (i & 1) * (32 * NC);
+                        const float ws = pick(other(i)) * inv;
+#pragma unroll
+                        for (int c = 0; c < NC; ++c) {
+                            const float4 val = buf[lane * NC + (c ^ (lane & (NC - 1)))];
+                            if (ws != 0.f) {                     // an empty part may hold anything
+                                acc[4 * c] += ws * val.x;
+                                acc[4 * c + 1] += ws * val.y;
+                                acc[4 * c + 2] += ws * val.z;
+                                acc[4 * c + 3] += ws * val.w;
+                            }
+                        }
+                        __syncwarp();
+                        if (i + 2 < n_pairs) issue(i + 2);
+                    }
+                    if (row_ok) {
+#pragma unroll
+                        for (int q8 = 0; q8 < DH / 8; ++q8) {
+                            uint4 o4;
+                            o4.x = pack_bf16(acc[q8 * 8 + 0], acc[q8 * 8 + 1]);
+                            o4.y = pack_bf16(acc[q8 * 8 + 2], acc[q8 * 8 + 3]);
+                            o4.z = pack_bf16(acc[q8 * 8 + 4], acc[q8 * 8 + 5]);
+                            o4.w = pack_bf16(acc[q8 * 8 + 6], acc[q8 * 8 + 7]);
+                            *reinterpret_cast<uint4*>(dst + h * DH + q8 * 8) = o4;
+                        }
+                    }
+                }
             }
         }
     } else if (warp_u < TC_MMA_WARP) {
@@ -490,6 +619,8 @@ template <int D>
 static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_max, cudaStream_t st, int* nsplit_out) {
     const int R = p.l_C * p.G;
     const int row_tiles = (R + TC_ROWS - 1) / TC_ROWS;
+    p.Rp = (R + 1) & ~1;
+    if ((size_t)B * p.HG * row_tiles > ctx->att_count_elems) return cudaErrorNotSupported;
     constexpr int smem = 2 * 128 * D * 2 + 2 * TC_STAGES * TC_BN * D * 2 + 1024;
     cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -509,7 +640,7 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     int best = 1;
     double best_cost = 1e30;
     for (int ns = 1; ns <= kAttPrefillSplits && ns <= n_tiles; ++ns) {
-        if ((size_t)B * p.HG * ns * R * (D + 2) > ctx->att_part_elems) break;
+        if ((size_t)B * p.HG * ns * p.Rp * (D + 2) > ctx->att_part_elems) break;
         const int per = (n_tiles + ns - 1) / ns;
         const int waves = (ctas * ns + ctx->num_sms - 1) / ctx->num_sms;
         const double cost = (double)waves * (per + 1.0) + (ns > 1 ? 0.5 * ns : 0.0);
@@ -526,12 +657,13 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
 }
 
 // Returns cudaErrorNotSupported when this path does not cover the shape (the caller then
-// uses the split kernel); nsplit_out tells the caller whether a merge pass must follow.
+// uses the split kernel); nsplit_out reports how many ways the key list was split (merged in-kernel).
 cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* K,
                              const __nv_bfloat16* V, const SeqMeta& meta, const int32_t* idx, const int32_t* n_sel,
                              __nv_bfloat16* O, int n_att_max, cudaStream_t st, int* nsplit_out) {
     TcAttendParams p;
     p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.status = ctx->status;
+    p.unit_count = ctx->att_count;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;

@@ -61,6 +61,8 @@ struct esa_ctx {
     uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys
     float* att_part;     // split-KV partial outputs + (m, l)
     size_t att_part_elems;
+    int* att_count;      // arrival counters of the split prefill attention, one per (sequence, kv head, row tile); 0 between launches
+    size_t att_count_elems;
     int* status;         // device status word
     int64_t launches;
     int last_lM[esa::kMaxBatch];
@@ -99,8 +101,8 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
                           const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
                           cudaStream_t st);
 
-// Prefill-sized chunks (l_C * H/H_G > kAttSplitRows) on tcgen05; *nsplit_out > 1 means partial
-// results were written to ctx->att_part and the merge kernel must follow.
+// Prefill-sized chunks (l_C * H/H_G > kAttSplitRows) on tcgen05; *nsplit_out reports the number of
+// key-list splits (their partials pass through ctx->att_part and are merged inside the kernel).
 cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
                              const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
                              const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
