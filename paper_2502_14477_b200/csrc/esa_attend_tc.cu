@@ -354,43 +354,78 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             // the row so that row-per-lane and row-per-half-warp accesses are both conflict-free.
             float4* stage = reinterpret_cast<float4*>(sQ + qt * Q_TILE_BYTES + (warp_u & 3) * (Q_TILE_BYTES / 4));
             const int wrow0 = row0 + qt * 128 + lane_base;        // first row of this warp
-            if (n_tiles > 0) {
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                    for (int cc = 0; cc < DH; cc += 32) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + h * DH + cc, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4)
-                            stage[lane * NC + ((cc / 4 + q4) ^ (lane & (NC - 1)))] =
-                                make_float4(__uint_as_float(o[4 * q4]), __uint_as_float(o[4 * q4 + 1]),
-                                            __uint_as_float(o[4 * q4 + 2]), __uint_as_float(o[4 * q4 + 3]));
-                    }
-                    __syncwarp();
-#pragma unroll 4
-                    for (int it = 0; it < NC; ++it) {
-                        const int e = it * 32 + lane, rr = e / NC, c = e % NC;
-                        const float4 val = stage[rr * NC + (c ^ (rr & (NC - 1)))];
-                        if (wrow0 + rr < R)
-                            __stcg(reinterpret_cast<float4*>(myO + (int64_t)(wrow0 + rr) * D + h * DH) + c, val);
-                    }
-                    __syncwarp();
-                }
-            }
-            if (row_ok) __stcg(reinterpret_cast<float2*>(myO + (int64_t)Rp * D) + row, make_float2(m_run, l_run));   // m = -inf: empty part
-            __threadfence();
+            int* cnt = p.unit_count + ((int64_t)b * p.HG + kvh) * gridDim.x + blockIdx.x;
+            // When every other CTA of the unit has arrived already, this one merges straight from its
+            // tensor memory and publishes nothing.
             asm volatile("bar.sync 1, 256;\n" ::: "memory");
             if (tid == 0) {
-                int* cnt = p.unit_count + ((int64_t)b * p.HG + kvh) * gridDim.x + blockIdx.x;
-                const int ticket = atomicAdd(cnt, 1);
-                if (ticket == p.nsplit - 1) *cnt = 0;          // ready for the next launch
-                merge_ticket = ticket;
+                const bool all_in = atomicAdd(cnt, 0) == p.nsplit - 1;
+                if (all_in) *cnt = 0;                              // ready for the next launch
+                merge_ticket = all_in ? p.nsplit - 1 : -1;
             }
             asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            if (merge_ticket != p.nsplit - 1) {
+                if (n_tiles > 0) {
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                        for (int cc = 0; cc < DH; cc += 32) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + h * DH + cc, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int q4 = 0; q4 < 8; ++q4)
+                                stage[lane * NC + ((cc / 4 + q4) ^ (lane & (NC - 1)))] =
+                                    make_float4(__uint_as_float(o[4 * q4]), __uint_as_float(o[4 * q4 + 1]),
+                                                __uint_as_float(o[4 * q4 + 2]), __uint_as_float(o[4 * q4 + 3]));
+                        }
+                        __syncwarp();
+#pragma unroll 4
+                        for (int it = 0; it < NC; ++it) {
+                            const int e = it * 32 + lane, rr = e / NC, c = e % NC;
+                            const float4 val = stage[rr * NC + (c ^ (rr & (NC - 1)))];
+                            if (wrow0 + rr < R)
+                                __stcg(reinterpret_cast<float4*>(myO + (int64_t)(wrow0 + rr) * D + h * DH) + c, val);
+                        }
+                        __syncwarp();
+                    }
+                }
+                if (row_ok) __stcg(reinterpret_cast<float2*>(myO + (int64_t)Rp * D) + row, make_float2(m_run, l_run));   // m = -inf: empty part
+                __threadfence();
+                asm volatile("bar.sync 1, 256;\n" ::: "memory");
+                if (tid == 0) {
+                    const int ticket = atomicAdd(cnt, 1);
+                    if (ticket == p.nsplit - 1) *cnt = 0;
+                    merge_ticket = ticket;
+                }
+                asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            }
             if (merge_ticket == p.nsplit - 1) {
                 __threadfence();
+                // The other parts' rows arrive through a ring of two shared-memory buffers per warp
+                // (16-byte cp.async, all copies of a buffer in flight together), in the order
+                // (column half, part).  The K/V stages serve as the ring: both warpgroups have passed
+                // their O_READY before the arrival barrier above, so no MMA reads them any more.
+                const int64_t own_off = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;     // this lane's row of O, in elements
+                const uint32_t own_lo = (uint32_t)own_off, own_hi = (uint32_t)(own_off >> 32);
+                float4* ring = reinterpret_cast<float4*>(sK + warp_u * (2 * TC_STAGES * KV_TILE_BYTES / 8));
+                const int n_other = p.nsplit - 1, n_pairs = 2 * n_other;
+                auto other = [&](int i) { const int s = i % n_other; return s + (s >= split ? 1 : 0); };
+                auto issue = [&](int i) {
+                    const int h = i / n_other;
+                    const float* srcO = unit_base + other(i) * part_stride + h * DH;
+                    float4* buf = ring + (i & 1) * (32 * NC);
+#pragma unroll
+                    for (int it = 0; it < NC; ++it) {
+                        const int e = it * 32 + lane, rr = e / NC, c = e % NC;
+                        const bool ok = wrow0 + rr < R;
+                        cp_async16(buf + rr * NC + (c ^ (rr & (NC - 1))), srcO + (int64_t)(ok ? wrow0 + rr : 0) * D + c * 4,
+                                   ok ? 16 : 0);
+                    }
+                    cp_async_commit();
+                };
+                issue(0);
+                if (n_pairs > 1) issue(1);
                 // weights of the parts in the log2 domain (Algorithm 1's merge of (O, m, l))
                 float w[kAttPrefillSplits];
                 float m_max = m_run;
@@ -411,29 +446,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 }
                 const float inv = 1.f / den;
                 auto pick = [&](int s) { return s == 0 ? w[0] : s == 1 ? w[1] : s == 2 ? w[2] : w[3]; };   // no dynamic register indexing
-                __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;
-                // The other parts' rows arrive through a ring of two shared-memory buffers per warp
-                // (16-byte cp.async, all copies of a buffer in flight together), in the order
-                // (column half, part).  The K/V stages serve as the ring: both warpgroups have passed
-                // their O_READY before the arrival barrier above, so no MMA reads them any more.
-                float4* ring = reinterpret_cast<float4*>(sK + warp_u * (2 * TC_STAGES * KV_TILE_BYTES / 8));
-                const int n_other = p.nsplit - 1, n_pairs = 2 * n_other;
-                auto other = [&](int i) { const int s = i % n_other; return s + (s >= split ? 1 : 0); };
-                auto issue = [&](int i) {
-                    const int h = i / n_other;
-                    const float* srcO = unit_base + other(i) * part_stride + h * DH;
-                    float4* buf = ring + (i & 1) * (32 * NC);
-#pragma unroll
-                    for (int it = 0; it < NC; ++it) {
-                        const int e = it * 32 + lane, rr = e / NC, c = e % NC;
-                        const bool ok = wrow0 + rr < R;
-                        cp_async16(buf + rr * NC + (c ^ (rr & (NC - 1))), srcO + (int64_t)(ok ? wrow0 + rr : 0) * D + c * 4,
-                                   ok ? 16 : 0);
-                    }
-                    cp_async_commit();
-                };
-                issue(0);
-                if (n_pairs > 1) issue(1);
 #pragma unroll 1
                 for (int h = 0; h < 2; ++h) {
                     float acc[DH];
@@ -469,16 +481,31 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                         __syncwarp();
                         if (i + 2 < n_pairs) issue(i + 2);
                     }
-                    if (row_ok) {
+                    // bf16 rows of this half leave through the staging buffer: 16-byte stores, whole rows per instruction
+                    {
+                        constexpr int NB = DH / 8;               // uint4 per staged row
+                        uint4* st16 = reinterpret_cast<uint4*>(stage);
 #pragma unroll
-                        for (int q8 = 0; q8 < DH / 8; ++q8) {
+                        for (int q8 = 0; q8 < NB; ++q8) {
                             uint4 o4;
                             o4.x = pack_bf16(acc[q8 * 8 + 0], acc[q8 * 8 + 1]);
                             o4.y = pack_bf16(acc[q8 * 8 + 2], acc[q8 * 8 + 3]);
                             o4.z = pack_bf16(acc[q8 * 8 + 4], acc[q8 * 8 + 5]);
                             o4.w = pack_bf16(acc[q8 * 8 + 6], acc[q8 * 8 + 7]);
-                            *reinterpret_cast<uint4*>(dst + h * DH + q8 * 8) = o4;
+                            st16[lane * NB + (q8 ^ (lane & (NB - 1)))] = o4;
                         }
+                        __syncwarp();
+#pragma unroll
+                        for (int it = 0; it < NB; ++it) {
+                            const int e = it * 32 + lane, rr = e / NB, c = e % NB;
+                            // lane rr of this warp owns row wrow0 + rr and knows where it goes
+                            const uint32_t lo = __shfl_sync(0xffffffffu, own_lo, rr), hi32 = __shfl_sync(0xffffffffu, own_hi, rr);
+                            if (wrow0 + rr < R) {
+                                __nv_bfloat16* d2 = p.O + (((int64_t)hi32 << 32) | lo) + h * DH;
+                                *reinterpret_cast<uint4*>(d2 + c * 8) = st16[rr * NB + (c ^ (rr & (NB - 1)))];
+                            }
+                        }
+                        __syncwarp();
                     }
                 }
             }
