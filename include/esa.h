@@ -65,7 +65,7 @@ typedef struct {
     int32_t l_init;        /* l_I                                                      */
     int32_t l_local;       /* l_L                                                      */
     int32_t top_k;         /* k                                                        */
-    int32_t eps;           /* proximity distance of Eq. 8, 0..16                       */
+    int32_t eps;           /* proximity distance of Eq. 8, 0..15                       */
     int32_t max_chunk;     /* largest l_C of any call                                  */
     int32_t max_batch;     /* largest B of any call, <= 64                             */
     int64_t max_tokens;    /* rows per sequence in every cache, < 2^31                 */

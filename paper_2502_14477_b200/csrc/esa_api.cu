@@ -18,7 +18,7 @@ bool config_ok(const esa_config* c) {
     if (c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->n_q_heads % c->n_kv_heads) return false;
     if (c->head_dim != 64 && c->head_dim != 128) return false;
     if (c->d_c != 32 && c->d_c != 64 && c->d_c != 128) return false;
-    if (c->l_init < 0 || c->l_local < 0 || c->top_k <= 0 || c->eps < 0 || c->eps > 16) return false;
+    if (c->l_init < 0 || c->l_local < 0 || c->top_k <= 0 || c->eps < 0 || c->eps > 15) return false;
     if (c->max_chunk <= 0 || c->max_batch <= 0 || c->max_batch > kMaxBatch) return false;
     if (c->max_tokens <= 0 || c->max_tokens >= (int64_t(1) << 31)) return false;
     if ((int64_t)c->n_q_heads * c->head_dim % 64 || (int64_t)c->n_kv_heads * c->head_dim % 64) return false;
@@ -242,6 +242,13 @@ esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, i
         map.row0[b] = (int)n_prev[b];
     }
     if (n_new == 0) return ESA_OK;
+    if (B * n_new <= kCompressGemvRows) {
+        cudaError_t e = launch_compress_gemv(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, ctx->Wk,
+                                             ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
+                                             ctx->cfg.max_tokens, map, nullptr, 0, (cudaStream_t)stream);
+        if (e != cudaErrorNotSupported) return from_cuda(e);
+        cudaGetLastError();
+    }
     if (ctx->has_wmaps) {
         cudaError_t e = launch_compress_tc(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, &ctx->wk_map,
                                            ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
@@ -292,7 +299,12 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
     e = cudaErrorNotSupported;
     bool rkey_cleared = false;
-    if (ctx->has_wmaps) {
+    if (B * l_C <= kCompressGemvRows) {
+        e = launch_compress_gemv(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
+                                 ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, ctx->rkey, B * l_C, st);
+        rkey_cleared = e == cudaSuccess;
+    }
+    if (e == cudaErrorNotSupported && ctx->has_wmaps) {
         // the compression kernel also clears the row-maximum words that the scoring pass accumulates into
         e = launch_compress_tc(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, &ctx->wq_map,
                                ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, ctx->rkey, B * l_C, st);

@@ -32,6 +32,7 @@ struct AttendParams {
     const int32_t* idx;       // [B, top_k]
     const int32_t* n_sel;     // [B]
     float* part;              // split partials
+    int* unit_count;          // arrival counters per (sequence, key/value head) for the in-kernel merge of the decode kernel
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
@@ -267,36 +268,30 @@ attend_kernel(AttendParams p) {
 // O = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with M = max_s m_s.
 // One warp per output row: each lane owns D / 32 consecutive columns, so a part's row is one
 // coalesced read and the result one coalesced bf16 write.
+// Combines the nsplit parts of one row (Algorithm 1's merge of (O, m, l)) and writes the bf16 row.
+// `base` points at the row's slot in part 0, parts are `sstride` floats apart.  Loads go to L2
+// (the parts may have been written by other SMs a moment ago).
 template <int D>
-__global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
+__device__ __forceinline__ void merge_row(const float* base, int64_t sstride, int nsplit, int lane, __nv_bfloat16* dst_row) {
     constexpr int PER = D / 32;                  // columns per lane: 2 or 4
-    pdl_wait();
-    pdl_launch_dependents();
-    const int R = p.l_C * p.G;
-    const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int kvh = blockIdx.y, b = blockIdx.z;
-    if (row >= R) return;
-    const float* base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit * R + row) * (D + 2);
-    const int64_t sstride = (int64_t)R * (D + 2);
     // parts are taken four at a time so that their loads are in flight together
     float M = -INFINITY;
-    for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, __ldg(base + s * sstride + D));
+    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, __ldcg(base + s * sstride + D));
     float den = 0.f;
     float acc[PER];
 #pragma unroll
     for (int i = 0; i < PER; ++i) acc[i] = 0.f;
-    for (int s0 = 0; s0 < p.nsplit; s0 += 4) {
+    for (int s0 = 0; s0 < nsplit; s0 += 4) {
         float mm[4], ll[4];
         float2 v[4][PER / 2];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const bool in = s0 + j < p.nsplit;
+            const bool in = s0 + j < nsplit;
             const float* ps = base + (in ? s0 + j : 0) * sstride;
-            mm[j] = in ? __ldg(ps + D) : -INFINITY;
-            ll[j] = __ldg(ps + D + 1);
+            mm[j] = in ? __ldcg(ps + D) : -INFINITY;
+            ll[j] = __ldcg(ps + D + 1);
 #pragma unroll
-            for (int i = 0; i < PER / 2; ++i) v[j][i] = __ldg(reinterpret_cast<const float2*>(ps + lane * PER + 2 * i));
+            for (int i = 0; i < PER / 2; ++i) v[j][i] = __ldcg(reinterpret_cast<const float2*>(ps + lane * PER + 2 * i));
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -311,10 +306,23 @@ __global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
         }
     }
     const float inv = 1.f / den;
-    const int cq = row / p.G, g = row % p.G;
-    __nv_bfloat16* dst = p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * p.G + g) * D + lane * PER;
 #pragma unroll
-    for (int i = 0; i < PER; i += 2) *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+    for (int i = 0; i < PER; i += 2)
+        *reinterpret_cast<uint32_t*>(dst_row + lane * PER + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) attend_merge_kernel(AttendParams p) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int R = p.l_C * p.G;
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int kvh = blockIdx.y, b = blockIdx.z;
+    if (row >= R) return;
+    const float* base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit * R + row) * (D + 2);
+    const int cq = row / p.G, g = row % p.G;
+    merge_row<D>(base, (int64_t)R * (D + 2), p.nsplit, lane, p.O + (((int64_t)b * p.l_C + cq) * p.H + kvh * p.G + g) * D);
 }
 
 // ---------------------------------------------------------------------------
@@ -540,6 +548,27 @@ attend_decode_kernel(AttendParams p) {
             if (col == 0) { dst[D] = M; dst[D + 1] = lsum; }
         }
     }
+    if (p.nsplit > 1) {
+        // The CTA that completes a (sequence, key/value head) unit merges its parts: an arrival
+        // counter decides, nobody waits, and the counter returns to 0 for the next launch.
+        __shared__ int s_last;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            int* cnt = p.unit_count + b * p.HG + kvh;
+            const int ticket = atomicAdd(cnt, 1);
+            s_last = ticket == p.nsplit - 1;
+            if (s_last) *cnt = 0;
+        }
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            for (int g = warp; g < G; g += DEC_WARPS) {
+                const float* base = p.part + (((int64_t)b * p.HG + kvh) * p.nsplit * G + g) * (D + 2);
+                merge_row<D>(base, (int64_t)G * (D + 2), p.nsplit, lane, p.O + ((int64_t)b * p.H + kvh * G + g) * D);
+            }
+        }
+    }
 }
 
 template <int D, int G>
@@ -559,13 +588,10 @@ static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     while (nsplit > 1 && (size_t)B * p.HG * nsplit * G * (D + 2) > ctx->att_part_elems) --nsplit;
     if (nsplit < 1) nsplit = 1;
     p.nsplit = nsplit;
+    if ((size_t)B * p.HG > ctx->att_count_elems) return cudaErrorInvalidConfiguration;
+    p.unit_count = ctx->att_count;
     e = launch_pdl(attend_decode_kernel<D, G>, dim3(nsplit, p.HG, B), dim3(DEC_WARPS * 32), smem, st, p);
     ctx->launches += 1;
-    if (e != cudaSuccess) return e;
-    if (nsplit > 1) {
-        e = launch_pdl(attend_merge_kernel<D>, dim3((G + 7) / 8, p.HG, B), dim3(256), 0, st, p);
-        ctx->launches += 1;
-    }
     return e;
 }
 
@@ -617,7 +643,7 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
                           const __nv_bfloat16* V, const SeqMeta& meta, const int32_t* idx,
                           const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st) {
     AttendParams p;
-    p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part;
+    p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
@@ -754,7 +780,7 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
 
     AttendParams p;
     p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
-    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part;
+    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr;
     p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
     p.top_k = cfg->top_k; p.nsplit = 1;
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)D);

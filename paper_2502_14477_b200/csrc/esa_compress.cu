@@ -168,6 +168,85 @@ cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int row
 }
 
 // ---------------------------------------------------------------------------
+// Eq. 5 for a handful of rows (decode: one new token per sequence).  A GEMM tile would be
+// almost empty, so this is a GEMV: one CTA per output feature c.  Its threads split row c of W
+// into 16-byte chunks (one or two per thread, every load in flight at once: the kernel is a
+// single round trip to L2), form the partial dot products with every input row, and reduce
+// them through shuffles and shared memory.  fp32 accumulation, bias, one bf16 rounding.
+// ---------------------------------------------------------------------------
+constexpr int GEMV_ROWS = 8;        // input rows per pass
+constexpr int GEMV_THREADS = 256;
+
+__global__ void __launch_bounds__(GEMV_THREADS)
+compress_gemv_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
+                     const float* __restrict__ bias, __nv_bfloat16* __restrict__ dst, int rows, int rows_per_seq,
+                     int d_in, int dc, int64_t dst_seq_stride, RowMap map, uint32_t* zero_words, int zero_count) {
+    __shared__ float red[GEMV_THREADS / 32][GEMV_ROWS];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int c = blockIdx.x;                              // output feature of this CTA
+    const int r0 = blockIdx.y * GEMV_ROWS;                 // first input row of this pass
+    pdl_wait();
+    pdl_launch_dependents();
+    if (zero_words && blockIdx.x == 0 && blockIdx.y == 0)
+        for (int i = tid; i < zero_count; i += GEMV_THREADS) zero_words[i] = 0u;
+    const int nr = min(GEMV_ROWS, rows - r0);
+    float acc[GEMV_ROWS];
+#pragma unroll
+    for (int r = 0; r < GEMV_ROWS; ++r) acc[r] = 0.f;
+    const uint4* wrow = reinterpret_cast<const uint4*>(W + (int64_t)c * d_in);
+    const int chunks = d_in / 8;
+#pragma unroll 2
+    for (int ch = tid; ch < chunks; ch += GEMV_THREADS) {
+        const uint4 wv = __ldg(wrow + ch);
+        uint4 xv[GEMV_ROWS];
+#pragma unroll
+        for (int r = 0; r < GEMV_ROWS; ++r)
+            xv[r] = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)(r0 + min(r, nr - 1)) * d_in) + ch);
+        const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
+        float2 wf[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wf[i] = __bfloat1622float2(w2[i]);
+#pragma unroll
+        for (int r = 0; r < GEMV_ROWS; ++r) {
+            const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&xv[r]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 xf = __bfloat1622float2(x2[i]);
+                acc[r] = fmaf(wf[i].x, xf.x, acc[r]);
+                acc[r] = fmaf(wf[i].y, xf.y, acc[r]);
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < GEMV_ROWS; ++r) {
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) acc[r] += __shfl_xor_sync(0xffffffffu, acc[r], o);
+        if (lane == 0) red[warp][r] = acc[r];
+    }
+    __syncthreads();
+    if (tid < nr) {
+        float sum = bias ? bias[c] : 0.f;
+#pragma unroll
+        for (int w = 0; w < GEMV_THREADS / 32; ++w) sum += red[w][tid];
+        const int row = r0 + tid, b = row / rows_per_seq, i = row % rows_per_seq;
+        dst[((int64_t)b * dst_seq_stride + map.row0[b] + i) * dc + c] = __float2bfloat16_rn(sum);
+    }
+}
+
+cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
+                                 const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
+                                 int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
+                                 cudaStream_t st) {
+    const int rows = B * rows_per_seq;
+    if (rows > kCompressGemvRows || d_in % 8 != 0) return cudaErrorNotSupported;
+    const dim3 grid(ctx->dc, (rows + GEMV_ROWS - 1) / GEMV_ROWS);
+    cudaError_t e = launch_pdl(compress_gemv_kernel, grid, dim3(GEMV_THREADS), 0, st, X, W, bias, dst, rows,
+                               rows_per_seq, d_in, ctx->dc, dst_seq_stride, map, zero_words, zero_count);
+    ctx->launches += 1;
+    return e;
+}
+
+// ---------------------------------------------------------------------------
 // K/V cache append: rows of the chunk copied into the caller's caches.
 // ---------------------------------------------------------------------------
 __global__ void append_kv_kernel(const uint4* __restrict__ K_new, const uint4* __restrict__ V_new,

@@ -31,6 +31,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 constexpr int kAttMaxSplits = 64;     // split-KV factor of the attention kernel (small chunks)
 constexpr int kAttSplitRows = 64;     // split-KV is used only when l_C * (H/H_G) <= this
 constexpr int kAttPrefillSplits = 4; // largest split of a prefill-sized chunk's key list
+constexpr int kCompressGemvRows = 16;   // at most this many input rows (B * n_new): compression runs as a GEMV
 constexpr int kCompressMaxRows = 4096;
 
 // Destination rows of a compression: row i of sequence b goes to
@@ -119,6 +120,12 @@ bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, i
 
 // Eq. 5 on tcgen05 for d' in {64, 128} and d_in a multiple of 128.  X is [rows, d_in] contiguous.
 // cudaErrorNotSupported when the shape is not covered (the caller then uses the mma.sync kernel).
+// Compression of a handful of rows (B * rows_per_seq <= kCompressGemvRows) as a GEMV; optionally clears
+// zero_count words at zero_words.  cudaErrorNotSupported when the shape is not covered.
+cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
+                                 const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
+                                 int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
+                                 cudaStream_t st);
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
                                int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,

@@ -318,3 +318,8 @@ def test_argument_errors_leave_outputs_untouched():
     assert e.value.status == 7
     with pytest.raises(esa.EsaError):
         esa.Esa(esa.EsaConfig(7, 2, 64, 32, 4, 512, 256, 3, 128, 1, 1024))   # H not a multiple of H_G
+    # the pooling window of Eq. 8 is taken inside one warp: 2 * eps + 1 <= 31
+    with pytest.raises(esa.EsaError) as e:
+        esa.Esa(esa.EsaConfig(cfg.H, cfg.H_G, cfg.d, cfg.d_c, 4, 512, 256, 16, 128, 1, 1024))
+    assert e.value.status == 2
+    esa.Esa(esa.EsaConfig(cfg.H, cfg.H_G, cfg.d, cfg.d_c, 4, 512, 256, 15, 128, 1, 1024))
