@@ -22,6 +22,8 @@ namespace esa {
 constexpr int SEL_CLUSTER_MAX = 16;   // CTAs working on one sequence: 8, or 16 (beyond the portable size) for small batches
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_BINS = 2048;
+constexpr size_t kSelMinDynSmem = 100 * 1024;   // with the static 33 KB: more than half an SM's shared memory
+static_assert(SEL_CLUSTER_MAX <= 32, "one lane per lower-ranked CTA in the compaction");
 
 struct SelectParams {
     const uint32_t* skey;   // aggregated keys, or raw fp32 S when raw != 0
@@ -254,11 +256,19 @@ select_topk_kernel(SelectParams p) {
         if (lane == 31) { cta_cnt[0] = gi; cta_cnt[1] = ei; }
     }
     cluster.sync();
-    uint32_t gt_before = warp_cnt[0][warp], eq_before = warp_cnt[1][warp];
-    for (int r = 0; r < rank; ++r) {
-        gt_before += *cluster.map_shared_rank(&cta_cnt[0], r);
-        eq_before += *cluster.map_shared_rank(&cta_cnt[1], r);
+    // counts of the lower-ranked CTAs: one remote read per lane, all in flight together
+    uint32_t gt_before = 0, eq_before = 0;
+    if (lane < rank) {
+        gt_before = *cluster.map_shared_rank(&cta_cnt[0], lane);
+        eq_before = *cluster.map_shared_rank(&cta_cnt[1], lane);
     }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        gt_before += __shfl_xor_sync(0xffffffffu, gt_before, o);
+        eq_before += __shfl_xor_sync(0xffffffffu, eq_before, o);
+    }
+    gt_before += warp_cnt[0][warp];
+    eq_before += warp_cnt[1][warp];
     int32_t* out = p.idx_out + (int64_t)b * p.top_k;
     for (int m0 = w_lo; m0 < w_hi; m0 += 32) {
         int m = m0 + lane;
@@ -309,14 +319,14 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
-    // 16 CTAs per sequence while the whole batch still fits the machine at once and the device can
-    // place such a cluster; else the portable 8
+    // 16 CTAs per sequence while the whole batch still fits half the machine and the device can
+    // place such a cluster; 10 for somewhat larger batches; else the portable 8
     static int can16 = -1;
     if (can16 < 0) {
         cudaLaunchConfig_t probe = {};
         probe.gridDim = dim3(SEL_CLUSTER_MAX, 1);
         probe.blockDim = dim3(SEL_THREADS);
-        probe.dynamicSmemBytes = 0;
+        probe.dynamicSmemBytes = kSelMinDynSmem;
         cudaLaunchAttribute pa[1];
         pa[0].id = cudaLaunchAttributeClusterDimension;
         pa[0].val.clusterDim.x = SEL_CLUSTER_MAX;
@@ -328,13 +338,20 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
         can16 = (cudaOccupancyMaxActiveClusters(&n, select_topk_kernel, &probe) == cudaSuccess && n > 0) ? 1 : 0;
         if (!can16) cudaGetLastError();
     }
-    const int n_ctas = (can16 && B * SEL_CLUSTER_MAX <= ctx->num_sms / 2) ? SEL_CLUSTER_MAX : 8;
+    // (measured on 148 SMs with 8 sequences: clusters of 10 beat 8 by a few percent, clusters of 12 or 16 place badly)
+    int n_ctas = 8;
+    if (can16 && B * SEL_CLUSTER_MAX <= ctx->num_sms / 2) n_ctas = SEL_CLUSTER_MAX;
+    else if (can16 && B * 10 * 5 <= ctx->num_sms * 3) n_ctas = 10;
     // dynamic shared memory for a CTA's slice of pooled keys (largest sequence of the call)
     const int rows32 = (max_lM + 31) / 32;
     const int slice = ((rows32 + n_ctas - 1) / n_ctas) * 32;
     size_t smem = (size_t)slice * 4;
     if (smem > 160 * 1024) smem = 0;
     p.slice_cap = (int)(smem / 4);
+    // One CTA per SM: the passes are bound by instruction issue, and two of these 1024-thread CTAs on
+    // one SM (their registers and small slices would allow it) run at half speed each while other SMs
+    // idle -- measured: the block scheduler does pack them.
+    if (smem < kSelMinDynSmem) smem = kSelMinDynSmem;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_ctas, B);
     cfg.blockDim = dim3(SEL_THREADS);

@@ -148,6 +148,13 @@ def test_gqa_group_of_seven_stage_isolated():
     _stage_isolated(cfg, 10000, 1, heads=None)
 
 
+def test_odd_row_count_through_the_split_merge():
+    # l_C * G odd and not a multiple of the row tile: the last row tile is ragged, the parts of the
+    # split key list are padded to an even row count, and the merging CTA skips the rows past the end
+    cfg = syn.get_config("c4").with_(S=8192, l_C=255, l_L=1024, k=1024)
+    _stage_isolated(cfg, 20 * 255, 255, heads=[0, 6, 13, 27], check_scores=False)
+
+
 def test_all_equal_scores_take_lowest_indices():
     """Identical compressed keys give identical scores: the first k middle tokens win."""
     cfg = syn.get_config("c1")
