@@ -29,7 +29,7 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, att, att_count, status, total;
+    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, ghist0, att, att_count, status, total;
     size_t att_elems, att_count_elems;
 };
 
@@ -46,6 +46,7 @@ Layout make_layout(const esa_config* c) {
     L.rkey = take(4 * (size_t)c->max_batch * c->max_chunk);
     L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
+    L.ghist0 = take(4 * (size_t)c->max_batch * 2048);
     const size_t G = c->n_q_heads / c->n_kv_heads;
     size_t rows = (size_t)c->max_chunk * G;
     if (rows > (size_t)kAttSplitRows) rows = kAttSplitRows;
@@ -159,6 +160,8 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->rkey = reinterpret_cast<uint32_t*>(base + L.rkey);
     c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
+    c->ghist0 = reinterpret_cast<uint32_t*>(base + L.ghist0);
+    c->last_decode = false;
     c->att_part = reinterpret_cast<float*>(base + L.att);
     c->att_part_elems = L.att_elems;
     c->att_count = reinterpret_cast<int*>(base + L.att_count);
@@ -245,7 +248,7 @@ esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, i
     if (B * n_new <= kCompressGemvRows) {
         cudaError_t e = launch_compress_gemv(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, ctx->Wk,
                                              ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
-                                             ctx->cfg.max_tokens, map, nullptr, 0, (cudaStream_t)stream);
+                                             ctx->cfg.max_tokens, map, nullptr, 0, nullptr, 0, (cudaStream_t)stream);
         if (e != cudaErrorNotSupported) return from_cuda(e);
         cudaGetLastError();
     }
@@ -298,11 +301,14 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     RowMap zero;
     for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
     e = cudaErrorNotSupported;
-    bool rkey_cleared = false;
+    bool rkey_cleared = false, ghist_cleared = false;
     if (B * l_C <= kCompressGemvRows) {
+        // (with one query per sequence the scoring kernel also accumulates first-digit histograms: cleared here too)
         e = launch_compress_gemv(ctx, (const __nv_bfloat16*)Q_cur, B, l_C, ctx->dH, ctx->Wq,
-                                 ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, ctx->rkey, B * l_C, st);
+                                 ctx->has_bq ? ctx->bq : nullptr, ctx->Qc, l_C, zero, ctx->rkey, B * l_C,
+                                 l_C == 1 ? ctx->ghist0 : nullptr, B * 2048, st);
         rkey_cleared = e == cudaSuccess;
+        ghist_cleared = rkey_cleared && l_C == 1;
     }
     if (e == cudaErrorNotSupported && ctx->has_wmaps) {
         // the compression kernel also clears the row-maximum words that the scoring pass accumulates into
@@ -320,7 +326,8 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     SeqMeta smeta = meta;
     for (int b = 0; b < B; ++b)
         if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
-    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, st);
+    ctx->last_decode = l_C == 1;
+    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, ghist_cleared, st);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
     e = launch_select(ctx, B, l_C, smeta, max_lM, idx_out, n_sel_out, st);
     return from_cuda(e);

@@ -180,7 +180,8 @@ constexpr int GEMV_THREADS = 256;
 __global__ void __launch_bounds__(GEMV_THREADS)
 compress_gemv_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W,
                      const float* __restrict__ bias, __nv_bfloat16* __restrict__ dst, int rows, int rows_per_seq,
-                     int d_in, int dc, int64_t dst_seq_stride, RowMap map, uint32_t* zero_words, int zero_count) {
+                     int d_in, int dc, int64_t dst_seq_stride, RowMap map, uint32_t* zero_words, int zero_count,
+                     uint32_t* zero2_words, int zero2_count) {
     __shared__ float red[GEMV_THREADS / 32][GEMV_ROWS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = blockIdx.x;                              // output feature of this CTA
@@ -189,6 +190,8 @@ compress_gemv_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* _
     pdl_launch_dependents();
     if (zero_words && blockIdx.x == 0 && blockIdx.y == 0)
         for (int i = tid; i < zero_count; i += GEMV_THREADS) zero_words[i] = 0u;
+    if (zero2_words && blockIdx.y == 0)
+        for (int i = blockIdx.x * GEMV_THREADS + tid; i < zero2_count; i += gridDim.x * GEMV_THREADS) zero2_words[i] = 0u;
     const int nr = min(GEMV_ROWS, rows - r0);
     float acc[GEMV_ROWS];
 #pragma unroll
@@ -236,12 +239,13 @@ compress_gemv_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* _
 cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                  const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
                                  int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
-                                 cudaStream_t st) {
+                                 uint32_t* zero2_words, int zero2_count, cudaStream_t st) {
     const int rows = B * rows_per_seq;
     if (rows > kCompressGemvRows || d_in % 8 != 0) return cudaErrorNotSupported;
     const dim3 grid(ctx->dc, (rows + GEMV_ROWS - 1) / GEMV_ROWS);
     cudaError_t e = launch_pdl(compress_gemv_kernel, grid, dim3(GEMV_THREADS), 0, st, X, W, bias, dst, rows,
-                               rows_per_seq, d_in, ctx->dc, dst_seq_stride, map, zero_words, zero_count);
+                               rows_per_seq, d_in, ctx->dc, dst_seq_stride, map, zero_words, zero_count, zero2_words,
+                               zero2_count);
     ctx->launches += 1;
     return e;
 }

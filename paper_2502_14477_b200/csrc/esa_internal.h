@@ -58,8 +58,10 @@ struct esa_ctx {
     float* bk;           // [dc]
     __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
     uint32_t* rkey;      // [max_batch * max_chunk] ordered keys of the row maxima r_c
-    uint32_t* skey;      // [max_batch, max_tokens] aggregated scores (ordered keys), or raw fp32 S (l_C = 1)
-    uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys
+    uint32_t* skey;      // [max_batch, max_tokens] aggregated scores (ordered keys); unused when l_C = 1
+    uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys (l_C = 1: of the pooled raw scores, r not yet subtracted)
+    uint32_t* ghist0;    // [max_batch, 2048] first-digit histograms of pkey, filled by the decode scoring kernel
+    bool last_decode;    // the last selection ran with l_C = 1 (pkey holds raw pooled scores)
     float* att_part;     // split-KV partial outputs + (m, l)
     size_t att_part_elems;
     int* att_count;      // arrival counters of the split prefill attention, one per (sequence, kv head, row tile); 0 between launches
@@ -79,9 +81,10 @@ cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int row
                             int64_t dst_seq_stride, const RowMap& map, cudaStream_t st);
 
 // Eq. 6 + Eq. 4: fills ctx->skey (and ctx->rkey) for the middle tokens of every sequence.
-// rkey_cleared: the caller's compression kernel has already zeroed ctx->rkey for this call.
+// l_C = 1: fills ctx->pkey (pooled raw scores), ctx->ghist0 and ctx->rkey instead.
+// rkey_cleared / ghist_cleared: the caller's compression kernel has already zeroed ctx->rkey / ctx->ghist0 for this call.
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                         const SeqMeta& meta, int max_lM, bool rkey_cleared, cudaStream_t st);
+                         const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st);
 
 // The same for chunks of >= 64 queries and d' in {64, 128} on tcgen05 with TMA-fed tiles; expects
 // ctx->rkey zeroed (pass 1 clears the part of ctx->skey that pass 2 accumulates into).  cudaErrorNotSupported when the shape is not covered.
@@ -121,11 +124,11 @@ bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, i
 // Eq. 5 on tcgen05 for d' in {64, 128} and d_in a multiple of 128.  X is [rows, d_in] contiguous.
 // cudaErrorNotSupported when the shape is not covered (the caller then uses the mma.sync kernel).
 // Compression of a handful of rows (B * rows_per_seq <= kCompressGemvRows) as a GEMV; optionally clears
-// zero_count words at zero_words.  cudaErrorNotSupported when the shape is not covered.
+// zero_count words at zero_words (one CTA) and zero2_count words at zero2_words (spread over the grid).  cudaErrorNotSupported when the shape is not covered.
 cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                  const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
                                  int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
-                                 cudaStream_t st);
+                                 uint32_t* zero2_words, int zero2_count, cudaStream_t st);
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
                                int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,

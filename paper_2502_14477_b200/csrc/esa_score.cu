@@ -182,31 +182,56 @@ score_pass_kernel(ScoreParams p) {
 }
 
 // ---------------------------------------------------------------------------
-// l_C = 1: S[m] = q' . k'_m as a streaming matrix-vector product.
+// l_C = 1: S[m] = q' . k'_m as a streaming matrix-vector product, with the front half of the
+// selection fused in.  With a single query, Eq. 4 is s_m = S_m - r (r = max_m S_m), and the
+// proximity pooling of Eq. 8 commutes with subtracting r (x -> fl(x - r) is monotone), so the
+// kernel pools the raw scores: P_j = max of S over [j - eps, j + eps] clipped to M.  It leaves
+//   * pkey[m]  = order-preserving key of P_m,
+//   * ghist0   = per-sequence histogram of the keys' top 11 bits (first radix digit of Eq. 2),
+//   * rkey[b]  = key of r (atomic max),
+// and the selection kernel finds the k-th largest P, maps the threshold through fl(. - r) and
+// compacts on fl(P_m - r): exactly the set that selecting on s' would give, ties included.
+// A CTA owns up to SD_TOKENS consecutive middle tokens (plus eps recomputed neighbours on each side),
+// so the window maxima come from shared memory and the histogram is flushed once per CTA.
 // ---------------------------------------------------------------------------
+constexpr int SD_TOKENS = 2048;
+constexpr int SD_HALO = 16;          // largest eps
+constexpr int SD_THREADS = 256;
+constexpr int SD_BINS = 2048;
+
 struct ScoreDecodeParams {
     const __nv_bfloat16* kc;
     const __nv_bfloat16* qc;    // [B, DC]
     uint32_t* rkey;             // [B]
-    float* sraw;                // [B, max_tokens]
+    uint32_t* pkey;             // [B, max_tokens] keys of the pooled raw scores
+    uint32_t* ghist0;           // [B, SD_BINS], zero on entry
     int64_t max_tokens;
+    int eps;
+    int chunk;                  // middle tokens per CTA: a multiple of SD_THREADS, at most SD_TOKENS
     SeqMeta meta;
 };
 
 template <int DC>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(SD_THREADS)
 score_decode_kernel(ScoreDecodeParams p) {
     constexpr int LPR = DC / 8;         // lanes per key row (16 bytes each)
     constexpr int RPW = 32 / LPR;       // rows per warp access
     constexpr int UNROLL = 4;
+    __shared__ float sS[SD_TOKENS + 2 * SD_HALO];
+    __shared__ uint32_t shist[SD_BINS];
+    __shared__ float smax[SD_THREADS / 32];
     pdl_wait();
     pdl_launch_dependents();
     const int b = blockIdx.y;
-    const int lane = threadIdx.x & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int i_end = p.meta.i_end[b];
     const int l_M = p.meta.m_end[b] - i_end;
+    const int a = blockIdx.x * p.chunk;                // first middle token of this CTA
+    if (a >= l_M) return;
+    const int nb = min(p.chunk, l_M - a);
+    const int eps = p.eps;
     const uint4* kc = reinterpret_cast<const uint4*>(p.kc + ((int64_t)b * p.max_tokens + i_end) * DC);
-    float* out = p.sraw + (int64_t)b * p.max_tokens;
+    for (int i = tid; i < SD_BINS; i += SD_THREADS) shist[i] = 0u;
 
     float q[8];
     {
@@ -219,16 +244,16 @@ score_decode_kernel(ScoreDecodeParams p) {
             q[2 * i + 1] = f.y;
         }
     }
+    // scores of the tokens [lo, hi): this CTA's own and the neighbours its windows reach
+    const int lo = max(0, a - eps), hi = min(l_M, a + nb + eps);
     const int sub = lane / LPR, part = lane % LPR;
-    const int64_t warp_global = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     float vmax = -INFINITY;
-    for (int64_t base = warp_global * (RPW * UNROLL); base < l_M; base += n_warps * (RPW * UNROLL)) {
+    for (int base = lo + warp * (RPW * UNROLL); base < hi; base += (SD_THREADS / 32) * (RPW * UNROLL)) {
         uint4 v[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            int64_t m = base + u * RPW + sub;
-            v[u] = (m < l_M) ? __ldg(kc + m * LPR + part) : make_uint4(0, 0, 0, 0);
+            const int m = base + u * RPW + sub;
+            v[u] = (m < hi) ? __ldg(kc + (int64_t)m * LPR + part) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
@@ -242,42 +267,84 @@ score_decode_kernel(ScoreDecodeParams p) {
             }
 #pragma unroll
             for (int o = LPR / 2; o >= 1; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            int64_t m = base + u * RPW + sub;
-            if (m < l_M) {
-                if (part == 0) out[m] = acc;
+            const int m = base + u * RPW + sub;
+            if (m < hi) {
+                if (part == 0) sS[m - (a - eps)] = acc;
                 vmax = fmaxf(vmax, acc);
             }
         }
     }
+    // window positions outside M never win
+    for (int i = tid; i < nb + 2 * eps; i += SD_THREADS) {
+        const int m = a - eps + i;
+        if (m < 0 || m >= l_M) sS[i] = -INFINITY;
+    }
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, o));
-    __shared__ float smax[8];
-    if (lane == 0) smax[threadIdx.x >> 5] = vmax;
+    if (lane == 0) smax[warp] = vmax;
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         float v = smax[0];
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) v = fmaxf(v, smax[w]);
+        for (int w = 1; w < SD_THREADS / 32; ++w) v = fmaxf(v, smax[w]);
         if (v > -INFINITY) atomicMax(p.rkey + b, f32_to_key(v));
+    }
+    // Eq. 8 on the raw scores, keys, first radix digit
+    uint32_t* pk = p.pkey + (int64_t)b * p.max_tokens + a;
+    float best[SD_TOKENS / SD_THREADS];
+#pragma unroll
+    for (int qd = 0; qd < SD_TOKENS / SD_THREADS; ++qd) best[qd] = -INFINITY;
+    for (int w = 0; w <= 2 * eps; ++w) {
+#pragma unroll
+        for (int qd = 0; qd < SD_TOKENS / SD_THREADS; ++qd) {
+            const int i = min(qd * SD_THREADS + tid, nb - 1);          // clamped lanes are not stored
+            best[qd] = fmaxf(best[qd], sS[i + w]);
+        }
+    }
+#pragma unroll
+    for (int qd = 0; qd < SD_TOKENS / SD_THREADS; ++qd) {
+        const int i = qd * SD_THREADS + tid;
+        const bool valid = i < nb;
+        const uint32_t key = f32_to_key(best[qd]);
+        if (valid) pk[i] = key;
+        // aggregated over the warp: neighbouring tokens crowd into a few bins
+        const uint32_t peers = __match_any_sync(0xffffffffu, valid ? (key >> 21) : 0xffffffffu);
+        if (valid && lane == __ffs(peers) - 1) atomicAdd(&shist[key >> 21], (uint32_t)__popc(peers));
+    }
+    __syncthreads();
+    uint32_t* gh = p.ghist0 + (int64_t)b * SD_BINS;
+    for (int i = tid; i < SD_BINS; i += SD_THREADS) {
+        const uint32_t c = shist[i];
+        if (c) atomicAdd(gh + i, c);
     }
 }
 
 template <int DC>
 static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                                  const SeqMeta& meta, int max_lM, bool rkey_cleared, cudaStream_t st) {
+                                  const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st) {
     cudaError_t e = cudaSuccess;
     if (!rkey_cleared) e = cudaMemsetAsync(ctx->rkey, 0, sizeof(uint32_t) * (size_t)B * l_C, st);
     if (e != cudaSuccess) return e;
     if (l_C == 1) {
         ScoreDecodeParams p;
         p.kc = kc_cache; p.qc = ctx->Qc; p.rkey = ctx->rkey;
-        p.sraw = reinterpret_cast<float*>(ctx->skey);
-        p.max_tokens = ctx->cfg.max_tokens; p.meta = meta;
-        constexpr int rows_per_block = 8 * (32 / (DC / 8)) * 4;
-        int gx = (max_lM + rows_per_block - 1) / rows_per_block;
-        int cap = (8 * ctx->num_sms + B - 1) / B;
-        if (gx > cap) gx = cap;
+        p.pkey = ctx->pkey; p.ghist0 = ctx->ghist0;
+        p.max_tokens = ctx->cfg.max_tokens; p.eps = ctx->cfg.eps; p.meta = meta;
+        if (!ghist_cleared) {
+            e = cudaMemsetAsync(ctx->ghist0, 0, sizeof(uint32_t) * (size_t)B * SD_BINS, st);
+            if (e != cudaSuccess) return e;
+        }
+        // Long chunks: every CTA pays a serial start (clear) and tail (pooling, flush) that its loads do
+        // not cover.  Measured with 8 x 129k tokens: 256 / 512 / 1024 / 2048 tokens per CTA give
+        // 87 / 83 / 78 / 76 us for the whole selection.  Short sequences get shorter chunks so that
+        // there are still a few CTAs per SM.
+        int64_t chunk = ((int64_t)B * max_lM * 2 + 7 * ctx->num_sms - 1) / (7 * ctx->num_sms);
+        chunk = (chunk + SD_THREADS - 1) / SD_THREADS * SD_THREADS;
+        if (chunk > SD_TOKENS) chunk = SD_TOKENS;
+        if (chunk < SD_THREADS) chunk = SD_THREADS;
+        p.chunk = (int)chunk;
+        int gx = (max_lM + p.chunk - 1) / p.chunk;
         if (gx < 1) gx = 1;
-        e = launch_pdl(score_decode_kernel<DC>, dim3(gx, B), dim3(256), 0, st, p);
+        e = launch_pdl(score_decode_kernel<DC>, dim3(gx, B), dim3(SD_THREADS), 0, st, p);
         ctx->launches += 1;
         return e;
     }
@@ -311,11 +378,11 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
 }
 
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache, const SeqMeta& meta,
-                         int max_lM, bool rkey_cleared, cudaStream_t st) {
+                         int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st) {
     switch (ctx->dc) {
-        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
-        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
-        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, st);
+        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
+        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
+        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
     }
     return cudaErrorInvalidValue;
 }

@@ -26,25 +26,21 @@ constexpr size_t kSelMinDynSmem = 100 * 1024;   // with the static 33 KB: more t
 static_assert(SEL_CLUSTER_MAX <= 32, "one lane per lower-ranked CTA in the compaction");
 
 struct SelectParams {
-    const uint32_t* skey;   // aggregated keys, or raw fp32 S when raw != 0
-    const uint32_t* rkey;   // [B * l_C] (raw mode reads r of query 0)
-    uint32_t* pkey;         // pooled keys out
+    const uint32_t* skey;   // aggregated keys (unused when pooled != 0)
+    const uint32_t* rkey;   // [B * l_C] (pooled mode reads r of query 0)
+    uint32_t* pkey;         // pooled keys: out, or in when pooled != 0
+    const uint32_t* ghist0; // [B, SEL_BINS] first-digit histograms of pkey (pooled mode)
     int32_t* idx_out;       // [B, top_k]
     int32_t* n_sel_out;     // [B]
     int64_t max_tokens;
     int top_k;
     int eps;
-    int raw;
+    int pooled;             // the scoring kernel already pooled (keys of P = pooled raw scores) and took the first histogram
     int l_C;
     int slice_cap;          // keys of a CTA's slice that fit in its dynamic shared memory (0: none)
     SeqMeta meta;
 };
 
-__device__ __forceinline__ uint32_t load_agg_key(const uint32_t* src, int m, int raw, float r0) {
-    uint32_t v = src[m];
-    if (raw) return f32_to_key(__uint_as_float(v) - r0);
-    return v;
-}
 
 // Histogram update aggregated over the warp: pooled scores crowd into a handful of bins
 // (same sign and exponent), so lanes with equal bins elect one leader that adds their count.
@@ -130,7 +126,7 @@ select_topk_kernel(SelectParams p) {
 
     const uint32_t* src = p.skey + (int64_t)b * p.max_tokens;
     uint32_t* pk = p.pkey + (int64_t)b * p.max_tokens;
-    const int raw = p.raw;
+    const int pooled = p.pooled;
 
     // slice of this CTA: whole 32-element rows, contiguous
     const int rows32 = (l_M + 31) / 32;
@@ -145,7 +141,7 @@ select_topk_kernel(SelectParams p) {
     cluster.sync();     // every CTA's histograms are zero before anyone adds to them remotely
     pdl_wait();         // the scores come from the preceding kernel
     pdl_launch_dependents();
-    const float r0 = raw ? key_to_f32(p.rkey[(int64_t)b * p.l_C]) : 0.f;
+    const float r0 = pooled ? key_to_f32(p.rkey[(int64_t)b * p.l_C]) : 0.f;
 
     // ---- digit 0: pool (Eq. 8), store pooled keys, histogram of bits 31..21
     // A warp loads 32 consecutive keys starting eps before its first output and slides the
@@ -155,7 +151,26 @@ select_topk_kernel(SelectParams p) {
     // Later passes re-read the slice: from shared memory when it fits, else from pkey (L2).
     const bool in_smem = (hi - lo) <= p.slice_cap;
     const uint32_t* keys = in_smem ? slice_keys : pk + lo;     // keys[i] = s' of token lo + i
-    {
+    if (pooled) {
+        // the scoring kernel left the pooled keys and their first-digit histogram: fetch this CTA's slice
+        // (four independent loads per thread and round) and every CTA's copy of the histogram
+        if (in_smem) {
+            for (int i0 = 0; i0 < hi - lo; i0 += 4 * SEL_THREADS) {
+                uint32_t v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * SEL_THREADS + tid;
+                    v[u] = (i < hi - lo) ? __ldcg(pk + lo + i) : 0u;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + u * SEL_THREADS + tid;
+                    if (i < hi - lo) slice_keys[i] = v[u];
+                }
+            }
+        }
+        for (int i = tid; i < SEL_BINS; i += SEL_THREADS) ghist[0][i] = __ldcg(p.ghist0 + (int64_t)b * SEL_BINS + i);
+    } else {
         const int eps = p.eps;
         const int outs = 32 - 2 * eps;
         constexpr int UN = 4;                                   // independent loads in flight per lane
@@ -165,7 +180,7 @@ select_topk_kernel(SelectParams p) {
 #pragma unroll
             for (int u = 0; u < UN; ++u) {
                 const int mload = first0 + u * step - eps + lane;
-                key[u] = (first0 + u * step < hi && mload >= 0 && mload < l_M) ? load_agg_key(src, mload, raw, r0) : 0u;
+                key[u] = (first0 + u * step < hi && mload >= 0 && mload < l_M) ? src[mload] : 0u;
             }
 #pragma unroll
             for (int u = 0; u < UN; ++u) {
@@ -193,13 +208,15 @@ select_topk_kernel(SelectParams p) {
         __syncthreads();
         // all-reduce of the digit histogram: every non-empty local bin is added to every CTA's copy
         const int nb = 1 << nbits[pass];
-        for (int i = tid; i < nb; i += SEL_THREADS) {
-            const uint32_t c = hist[i];
-            if (c) {
-                for (int r = 0; r < n_ctas; ++r) atomicAdd(cluster.map_shared_rank(&ghist[pass][i], r), c);
+        if (!(pooled && pass == 0)) {      // (pooled: the first digit's histogram came complete from global memory)
+            for (int i = tid; i < nb; i += SEL_THREADS) {
+                const uint32_t c = hist[i];
+                if (c) {
+                    for (int r = 0; r < n_ctas; ++r) atomicAdd(cluster.map_shared_rank(&ghist[pass][i], r), c);
+                }
             }
+            cluster.sync();
         }
-        cluster.sync();
         find_bin(ghist[pass], nb, krem, scan_tmp, sh_found);
         prefix |= sh_found[0] << shifts[pass];
         krem = sh_found[1];
@@ -218,7 +235,11 @@ select_topk_kernel(SelectParams p) {
             if (take) hist_add(hist, (key >> sh) & dmask, active);
         }
     }
-    const uint32_t T = prefix;   // k-th largest key; krem of the keys equal to T are taken
+    // k-th largest key.  Pooled mode: the keys so far are those of P (raw pooled scores); Eq. 4's
+    // s' = fl(P - r) is a monotone map of P, so its k-th largest value is the image of the k-th
+    // largest P, and the compaction below runs on the mapped keys (ties of s' included).
+    const uint32_t T = pooled ? f32_to_key(key_to_f32(prefix) - r0) : prefix;
+    auto final_key = [&](uint32_t key) { return pooled ? f32_to_key(key_to_f32(key) - r0) : key; };
 
     // ---- ordered compaction
     // each warp owns a contiguous run of 32-element rows of the CTA's slice
@@ -228,7 +249,7 @@ select_topk_kernel(SelectParams p) {
     const int w_hi = min(hi, lo + (warp + 1) * rows_per_warp * 32);
     uint32_t n_gt = 0, n_eq = 0;
     for (int m = w_lo + lane; m < w_hi; m += 32) {
-        uint32_t key = keys[m - lo];
+        uint32_t key = final_key(keys[m - lo]);
         n_gt += key > T;
         n_eq += key == T;
     }
@@ -257,22 +278,27 @@ select_topk_kernel(SelectParams p) {
     }
     cluster.sync();
     // counts of the lower-ranked CTAs: one remote read per lane, all in flight together
-    uint32_t gt_before = 0, eq_before = 0;
-    if (lane < rank) {
-        gt_before = *cluster.map_shared_rank(&cta_cnt[0], lane);
-        eq_before = *cluster.map_shared_rank(&cta_cnt[1], lane);
+    uint32_t gt_before = 0, eq_before = 0, gt_all = 0;
+    if (lane < n_ctas) {
+        gt_all = *cluster.map_shared_rank(&cta_cnt[0], lane);
+        if (lane < rank) {
+            gt_before = gt_all;
+            eq_before = *cluster.map_shared_rank(&cta_cnt[1], lane);
+        }
     }
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) {
         gt_before += __shfl_xor_sync(0xffffffffu, gt_before, o);
         eq_before += __shfl_xor_sync(0xffffffffu, eq_before, o);
+        gt_all += __shfl_xor_sync(0xffffffffu, gt_all, o);
     }
+    krem = (uint32_t)k - gt_all;      // keys equal to T still to take (= the radix passes' remainder; recounted for the mapped keys)
     gt_before += warp_cnt[0][warp];
     eq_before += warp_cnt[1][warp];
     int32_t* out = p.idx_out + (int64_t)b * p.top_k;
     for (int m0 = w_lo; m0 < w_hi; m0 += 32) {
         int m = m0 + lane;
-        uint32_t key = (m < w_hi) ? keys[m - lo] : 0u;
+        uint32_t key = (m < w_hi) ? final_key(keys[m - lo]) : 0u;
         bool gt = (m < w_hi) && key > T;
         bool eq = (m < w_hi) && key == T;
         uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
@@ -303,9 +329,11 @@ __global__ void select_all_kernel(int32_t* idx_out, int32_t* n_sel_out, int top_
     if (blockIdx.x == 0 && threadIdx.x == 0) n_sel_out[b] = n;
 }
 
-__global__ void read_pooled_kernel(const uint32_t* __restrict__ pkey, float* __restrict__ dst, int64_t n) {
+// r: key of the row maximum to subtract (decode: pkey holds the pooled raw scores), or null
+__global__ void read_pooled_kernel(const uint32_t* __restrict__ pkey, const uint32_t* __restrict__ r,
+                                   float* __restrict__ dst, int64_t n) {
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) dst[i] = key_to_f32(pkey[i]);
+    if (i < n) dst[i] = r ? key_to_f32(pkey[i]) - key_to_f32(*r) : key_to_f32(pkey[i]);
 }
 
 cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, int32_t* idx_out,
@@ -314,7 +342,7 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     p.skey = ctx->skey; p.rkey = ctx->rkey; p.pkey = ctx->pkey;
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.top_k = ctx->cfg.top_k; p.eps = ctx->cfg.eps;
-    p.raw = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
+    p.pooled = (l_C == 1) ? 1 : 0; p.ghist0 = ctx->ghist0; p.l_C = l_C; p.meta = meta;
     cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
@@ -384,7 +412,7 @@ cudaError_t launch_select_all(esa_ctx* ctx, int B, const SeqMeta& meta, int32_t*
 
 cudaError_t launch_read_pooled(esa_ctx* ctx, int b, float* dst_dev, int64_t n, cudaStream_t st) {
     read_pooled_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ctx->pkey + (int64_t)b * ctx->cfg.max_tokens,
-                                                                   dst_dev, n);
+                                                                   ctx->last_decode ? ctx->rkey + b : nullptr, dst_dev, n);
     ctx->launches += 1;
     return cudaGetLastError();
 }
