@@ -40,8 +40,8 @@ import esa_synth as syn
 N_LAYERS_STACK = 32
 # dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised in
 # profiles/dram_bytes_per_kernel.txt (same kernels, same launch shapes as the timed workloads).
-ATTEND_TC_DRAM_BYTES = 32504832 + 471296
-DECODE_STEP_DRAM_BYTES = (205785856 + 1053440) + 541184 + 39168 + 303104 + 1134848 + (264000256 + 3063552) + 4179456
+ATTEND_TC_DRAM_BYTES = 32079104 + 37888
+DECODE_STEP_DRAM_BYTES = (205819136 + 574464) + 39168 + 300288 + 1133056 + (264769536 + 140800) + 4243968
 
 
 # ----------------------------------------------------------------------------
@@ -413,7 +413,7 @@ def run_esa(args, cfg):
     att_ms = sum(a.elapsed_time(b) for (_, _, a, b) in events)
     att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
     achieved = att_flops / (att_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (+ attend_merge_kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
+    roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (key-list splits merged inside the kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": ATTEND_TC_DRAM_BYTES,
                 "traffic_unit": "bytes per attend_tc_kernel launch (ncu, profiles/dram_bytes_per_kernel.txt)",
                 "peak_source": peaks["source"] + " sustained bf16", "share_of_step": att_ms / (ms_total),
