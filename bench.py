@@ -178,13 +178,35 @@ def make_ctx(cfg, max_tokens, max_chunk, max_batch):
                                  max_chunk, max_batch, max_tokens))
 
 
+_SIDE = []
+
+
+def _side_stream():
+    if not _SIDE:
+        _SIDE.append(torch.cuda.Stream())
+    return _SIDE[0]
+
+
 def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
     """The whole chunked prefill of one layer with inputs resident in HBM."""
     Kc, idx, n_sel, O = bufs
+    # The compressed keys of the current chunk are not read by this chunk's selection (C is not
+    # part of M): esa_compress_keys runs on a side stream beside the attention, and the selection
+    # waits for the previous chunk's compression, which covers every row that M can contain.
+    main = torch.cuda.current_stream()
+    side = _side_stream()
+    side.wait_stream(main)
+    prev = None
     for t in range(0, cfg.S, cfg.l_C):
         l_C = min(cfg.l_C, cfg.S - t)
         Qc = L.Q[:, t: t + l_C]
-        ctx.compress_keys(L.K[:, t: t + l_C], Kc, [t])
+        with torch.cuda.stream(side):
+            ctx.compress_keys(L.K[:, t: t + l_C], Kc, [t])
+            done = torch.cuda.Event()
+            done.record(side)
+        if prev is not None:
+            main.wait_event(prev)
+        prev = done
         ctx.select(Qc, Kc, [t], idx, n_sel)
         if attend_events is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -193,6 +215,7 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
         if attend_events is not None:
             e1.record()
             attend_events.append((t, l_C, e0, e1))
+    main.wait_stream(side)
 
 
 def run_prefill_layer_e2e(ctx, cfg, L, bufs, caches, stage, O_host, streams):
@@ -332,11 +355,23 @@ def time_decode(cfg3, n_steps, rank_seed):
     n_sel = torch.zeros(B, dtype=torch.int32, device="cuda")
     O = torch.empty(B, 1, cfg3.H, cfg3.d, dtype=torch.bfloat16, device="cuda")
 
+    main = torch.cuda.current_stream()
+    side = _side_stream()
+    side.wait_stream(main)
+    prev = [None]
+
     def step(i):
+        # the new token's compressed key is not read by this step's selection: side stream
         t = [S + i] * B
         kn, vn = Knew[i], Vnew[i]
+        with torch.cuda.stream(side):
+            ctx.compress_keys(kn, Kc, t)
+            done = torch.cuda.Event()
+            done.record(side)
         ctx.append_kv(kn, vn, K, V, t)
-        ctx.compress_keys(kn, Kc, t)
+        if prev[0] is not None:
+            main.wait_event(prev[0])
+        prev[0] = done
         ctx.select(Qs[i], Kc, t, idx, n_sel)
         ctx.attend(Qs[i], K, V, t, idx, n_sel, O)
 
@@ -348,6 +383,7 @@ def time_decode(cfg3, n_steps, rank_seed):
     e0.record()
     for i in range(n_steps):
         step(i)
+    main.wait_stream(side)
     e1.record()
     torch.cuda.synchronize()
     us = 1e3 * e0.elapsed_time(e1) / n_steps

@@ -26,8 +26,13 @@
  *   - *_async variants only enqueue work on the given CUDA stream (a cudaStream_t passed
  *     as void*) and return without synchronising.  The plain variants run on the legacy
  *     default stream and return after the work has finished.
- *   - A context owns device workspace shared by its calls: calls on the same context must
- *     be ordered (one stream, or externally synchronised).  Use one context per stream.
+ *   - A context owns device workspace shared by its calls: esa_select and esa_attend calls
+ *     on the same context must be ordered (one stream, or externally synchronised); use one
+ *     context per stream for them.  esa_compress_keys and esa_append_kv touch none of that
+ *     workspace (they read the weights and write caller memory): they may run on another
+ *     stream beside a select or attend of the same context, as long as the caller orders
+ *     them against the calls that read the rows they write (the selection reads rows of M
+ *     only, the attention reads every row up to the end of the current chunk).
  *   - Device-side problems (a bounded wait that ran out) are recorded in a status word
  *     read by esa_last_device_status; kernels never trap.
  *   - The compressed-key cache is caller memory with library-defined contents: row p of

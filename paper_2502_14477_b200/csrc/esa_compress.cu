@@ -258,6 +258,8 @@ __global__ void append_kv_kernel(const uint4* __restrict__ K_new, const uint4* _
                                  int row_chunks, int64_t max_tokens, RowMap map) {
     const int b = blockIdx.y;
     const int64_t per_seq = (int64_t)n_new * row_chunks;
+    pdl_wait();                 // the previous step's attention may still be reading the caches
+    pdl_launch_dependents();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < per_seq;
          i += (int64_t)gridDim.x * blockDim.x) {
         int64_t src = (int64_t)b * per_seq + i;
@@ -275,11 +277,12 @@ cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new, co
     int gx = (int)((per_seq + 255) / 256);
     if (gx > 4 * ctx->num_sms) gx = 4 * ctx->num_sms;
     if (gx < 1) gx = 1;
-    append_kv_kernel<<<dim3(gx, B), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(K_new), reinterpret_cast<const uint4*>(V_new),
-        reinterpret_cast<uint4*>(K_cache), reinterpret_cast<uint4*>(V_cache), n_new, row_chunks,
-        ctx->cfg.max_tokens, map);
+    cudaError_t e = launch_pdl(append_kv_kernel, dim3(gx, B), dim3(256), 0, st,
+                               reinterpret_cast<const uint4*>(K_new), reinterpret_cast<const uint4*>(V_new),
+                               reinterpret_cast<uint4*>(K_cache), reinterpret_cast<uint4*>(V_cache), n_new, row_chunks,
+                               ctx->cfg.max_tokens, map);
     ctx->launches += 1;
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
