@@ -448,34 +448,47 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 auto pick = [&](int s) { return s == 0 ? w[0] : s == 1 ? w[1] : s == 2 ? w[2] : w[3]; };   // no dynamic register indexing
 #pragma unroll 1
                 for (int h = 0; h < 2; ++h) {
+                    // The parts are added in split order whichever CTA happens to merge (its own part comes
+                    // from tensor memory, the others from the ring), so the result does not depend on the
+                    // order of arrival: the same bits as a merge pass over all parts.
                     float acc[DH];
-                    {
+#pragma unroll
+                    for (int i = 0; i < DH; ++i) acc[i] = 0.f;
+                    auto add_own = [&]() {
                         const float wo = pick(split) * inv;       // 0 when this CTA's own part is empty
 #pragma unroll
-                        for (int cc = 0; cc < DH; cc += 32) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + h * DH + cc, o);
+                        for (int cc = 0; cc < DH; cc += 16) {
+                            uint32_t o[16];
+                            tmem_ld16(tO + h * DH + cc, o);
                             tmem_wait_ld();
+                            if (wo != 0.f) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) acc[cc + i] = (wo == 0.f) ? 0.f : __uint_as_float(o[i]) * wo;
+                                for (int i = 0; i < 16; ++i) acc[cc + i] = fmaf(wo, __uint_as_float(o[i]), acc[cc + i]);
+                            }
                         }
-                    }
+                    };
+                    int k = 0;                                    // index among the other parts
 #pragma unroll 1
-                    for (int k = 0; k < n_other; ++k) {
+                    for (int sp = 0; sp < p.nsplit; ++sp) {
+                        if (sp == split) {
+                            add_own();
+                            continue;
+                        }
                         const int i = h * n_other + k;
+                        ++k;
                         if (i + 1 < n_pairs) cp_async_wait<1>();
                         else cp_async_wait<0>();
                         __syncwarp();
                         const float4* buf = ring + (i & 1) * (32 * NC);
-                        const float ws = pick(other(i)) * inv;
+                        const float ws = pick(sp) * inv;
 #pragma unroll
                         for (int c = 0; c < NC; ++c) {
                             const float4 val = buf[lane * NC + (c ^ (lane & (NC - 1)))];
                             if (ws != 0.f) {                     // an empty part may hold anything
-                                acc[4 * c] += ws * val.x;
-                                acc[4 * c + 1] += ws * val.y;
-                                acc[4 * c + 2] += ws * val.z;
-                                acc[4 * c + 3] += ws * val.w;
+                                acc[4 * c] = fmaf(ws, val.x, acc[4 * c]);
+                                acc[4 * c + 1] = fmaf(ws, val.y, acc[4 * c + 1]);
+                                acc[4 * c + 2] = fmaf(ws, val.z, acc[4 * c + 2]);
+                                acc[4 * c + 3] = fmaf(ws, val.w, acc[4 * c + 3]);
                             }
                         }
                         __syncwarp();

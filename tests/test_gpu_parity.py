@@ -303,6 +303,54 @@ def test_batch_of_ragged_sequences_dc64():
         hp.check_compressed(seq.Kc[b, : t], K64[:t].reshape(t, -1), Wk, what=f"ragged seq {b} cache")
 
 
+def test_compress_keys_on_a_side_stream_matches_the_serial_order():
+    """esa_compress_keys uses none of the context's workspace: run beside select/attend on another
+    stream (ordered only against the selection that first reads its rows) it must give the very
+    bits of the one-stream order."""
+    cfg = syn.get_config("c1")
+    n = 2048
+    outs = []
+    for use_side in (False, True):
+        ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=cfg.l_C, max_batch=1)
+        seq = hp.DeviceSeq(cfg, max_tokens=n, B=1)
+        seq.fill_kv(0, n)
+        O = torch.zeros(1, n, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda")
+        idx_log = []
+        main = torch.cuda.current_stream()
+        side = torch.cuda.Stream()
+        side.wait_stream(main)
+        prev = None
+        for t in range(0, n, cfg.l_C):
+            Q = seq.q_rows(t, t + cfg.l_C)
+            Knew = seq.K[:, t: t + cfg.l_C].contiguous()
+            if use_side:
+                side.wait_stream(main)          # Knew was produced on the main stream
+                with torch.cuda.stream(side):
+                    ctx.compress_keys(Knew, seq.Kc, [t])
+                    done = torch.cuda.Event()
+                    done.record(side)
+                Knew.record_stream(side)
+                if prev is not None:
+                    main.wait_event(prev)
+                prev = done
+            else:
+                ctx.compress_keys(Knew, seq.Kc, [t])
+            ctx.select(Q, seq.Kc, [t], seq.idx, seq.n_sel)
+            ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O[:, t: t + cfg.l_C])
+            idx_log.append((seq.idx.clone(), seq.n_sel.clone()))
+        main.wait_stream(side)
+        torch.cuda.synchronize()
+        assert ctx.last_device_status() == 0
+        outs.append((seq.Kc.clone(), O, idx_log))
+    (kc0, o0, l0), (kc1, o1, l1) = outs
+    assert torch.equal(kc0, kc1)
+    assert torch.equal(o0, o1)
+    for (i0, n0), (i1, n1) in zip(l0, l1):
+        assert torch.equal(n0, n1)
+        k = int(n0[0])
+        assert torch.equal(i0[0, :k], i1[0, :k])
+
+
 # ----------------------------------------------------------------- error paths
 def test_argument_errors_leave_outputs_untouched():
     import paper_2502_14477_b200 as esa
