@@ -196,17 +196,22 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
     main = torch.cuda.current_stream()
     side = _side_stream()
     side.wait_stream(main)
-    prev = None
+    done = []                                   # done[c]: rows of chunk c are compressed
     for t in range(0, cfg.S, cfg.l_C):
         l_C = min(cfg.l_C, cfg.S - t)
         Qc = L.Q[:, t: t + l_C]
         with torch.cuda.stream(side):
             ctx.compress_keys(L.K[:, t: t + l_C], Kc, [t])
-            done = torch.cuda.Event()
-            done.record(side)
-        if prev is not None:
-            main.wait_event(prev)
-        prev = done
+            ev = torch.cuda.Event()
+            ev.record(side)
+            done.append(ev)
+        # M = [i_end, m_end): the last chunk that reaches into it.  It was enqueued l_L tokens ago and has
+        # normally finished: then no wait is put between the attention and the next selection (a stream
+        # wait would keep the selection's first kernel from being set up under the attention's tail).
+        m_end = max(min(cfg.l_I, t), t - cfg.l_L)
+        c_need = (m_end + cfg.l_C - 1) // cfg.l_C - 1
+        if c_need >= 0 and not done[c_need].query():
+            main.wait_event(done[c_need])
         ctx.select(Qc, Kc, [t], idx, n_sel)
         if attend_events is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -358,20 +363,23 @@ def time_decode(cfg3, n_steps, rank_seed):
     main = torch.cuda.current_stream()
     side = _side_stream()
     side.wait_stream(main)
-    prev = [None]
+    done = {}                                   # done[i]: the compressed key of step i's token is in place
 
     def step(i):
-        # the new token's compressed key is not read by this step's selection: side stream
+        # the new token's compressed key is not read by this step's selection (it enters M l_L steps
+        # later): side stream, and a wait only for a step whose key is needed and not yet written
         t = [S + i] * B
         kn, vn = Knew[i], Vnew[i]
         with torch.cuda.stream(side):
             ctx.compress_keys(kn, Kc, t)
-            done = torch.cuda.Event()
-            done.record(side)
+            ev = torch.cuda.Event()
+            ev.record(side)
+            done[i] = ev
         ctx.append_kv(kn, vn, K, V, t)
-        if prev[0] is not None:
-            main.wait_event(prev[0])
-        prev[0] = done
+        need = i - cfg3.l_L - 1                 # last step whose token is inside M now
+        if need in done and not done[need].query():
+            main.wait_event(done[need])
+        done.pop(need - 1, None)
         ctx.select(Qs[i], Kc, t, idx, n_sel)
         ctx.attend(Qs[i], K, V, t, idx, n_sel, O)
 
