@@ -48,8 +48,8 @@ def run_step_gpu(ctx, seq: hp.DeviceSeq, Q: torch.Tensor, t_list, do_compress=Tr
 
 
 # --------------------------------------------------------------- compression
-@pytest.mark.parametrize("name,n_new,with_bias", [("c1", 128, False), ("c1", 37, True), ("c2", 512, False),
-                                                   ("c2", 1, False), ("c2", 700, True)])
+@pytest.mark.parametrize("name,n_new,with_bias", [("c1", 128, False), ("c1", 37, True), ("c1", 13, True), ("c1", 7, True), ("c1", 1, False), ("c2", 512, False),
+                                                   ("c2", 1, False), ("c2", 8, True), ("c2", 700, True)])
 def test_compress_keys_parity(name, n_new, with_bias):
     cfg = syn.get_config(name).with_(S=2048, n_decode=0)
     bias = syn.compressor_bias(cfg) if with_bias else None
