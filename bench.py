@@ -187,8 +187,17 @@ def _side_stream():
     return _SIDE[0]
 
 
-def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
-    """The whole chunked prefill of one layer with inputs resident in HBM."""
+ATTEND_EVENT_EVERY = 8      # one attention launch in this many carries CUDA events (see run_prefill_layer)
+
+
+def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None, phase=0):
+    """The whole chunked prefill of one layer with inputs resident in HBM.
+
+    attend_events: list that receives (t, l_C, start, end) CUDA events around attention launches.
+    An event record between two kernels keeps the second one from being set up under the first
+    one's tail (programmatic dependent launch), which costs 8 % of the step when every launch is
+    bracketed; so one launch in ATTEND_EVENT_EVERY is, the sampled position rotating with `phase`
+    (over 8 steps every chunk position is sampled once)."""
     Kc, idx, n_sel, O = bufs
     # The compressed keys of the current chunk are not read by this chunk's selection (C is not
     # part of M): esa_compress_keys runs on a side stream beside the attention, and the selection
@@ -213,11 +222,12 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None):
         if c_need >= 0 and not done[c_need].query():
             main.wait_event(done[c_need])
         ctx.select(Qc, Kc, [t], idx, n_sel)
-        if attend_events is not None:
+        timed = attend_events is not None and (t // cfg.l_C + phase) % ATTEND_EVENT_EVERY == 0
+        if timed:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
         ctx.attend(Qc, L.K, L.V, [t], idx, n_sel, O[:, t: t + l_C])
-        if attend_events is not None:
+        if timed:
             e1.record()
             attend_events.append((t, l_C, e0, e1))
     main.wait_stream(side)
@@ -429,7 +439,7 @@ def run_esa(args, cfg):
     def one_step(i, ev=None):
         L = layers[i % n_res]
         ctx.set_compressors(L.wq, None, L.wk, None)
-        run_prefill_layer(ctx, cfg, L, bufs, ev)
+        run_prefill_layer(ctx, cfg, L, bufs, ev, phase=i)
 
     for i in range(args.warmup):
         one_step(i)
@@ -455,13 +465,16 @@ def run_esa(args, cfg):
 
     # roofline of the dominant kernel (the attention launches), timed inside the region above
     att_ms = sum(a.elapsed_time(b) for (_, _, a, b) in events)
+    n_chunks = (cfg.S + cfg.l_C - 1) // cfg.l_C
     att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
     achieved = att_flops / (att_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (key-list splits merged inside the kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": ATTEND_TC_DRAM_BYTES,
                 "traffic_unit": "bytes per attend_tc_kernel launch (ncu, profiles/dram_bytes_per_kernel.txt)",
-                "peak_source": peaks["source"] + " sustained bf16", "share_of_step": att_ms / (ms_total),
-                "launches": len(events)}
+                "peak_source": peaks["source"] + " sustained bf16",
+                "share_of_step": att_ms * (args.steps * n_chunks / max(1, len(events))) / ms_total,
+                "launches": len(events),
+                "sampling": "CUDA events around 1 attention launch in %d, position rotating over the steps" % ATTEND_EVENT_EVERY}
 
     # end to end: host inputs and outputs
     L0 = layers[0]
