@@ -179,7 +179,8 @@ esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int6
 int64_t esa_launch_count(const esa_ctx* ctx);
 
 /* Synchronises the stream, then returns ESA_OK or the error a kernel recorded
- * (and clears the record). */
+ * (and clears the record, together with the merge bookkeeping that an abandoned
+ * kernel may have left behind: the context stays usable). */
 esa_status esa_last_device_status(esa_ctx* ctx, void* stream);
 
 #ifdef __cplusplus

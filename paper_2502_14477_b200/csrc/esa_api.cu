@@ -388,6 +388,8 @@ esa_status esa_last_device_status(esa_ctx* ctx, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return ESA_ERR_CUDA;
     if (h != 0) {
         if (cudaMemsetAsync(ctx->status, 0, sizeof(int), st) != cudaSuccess) return ESA_ERR_CUDA;
+        // a kernel that gave up may have left arrival counters of the in-kernel merges behind
+        if (cudaMemsetAsync(ctx->att_count, 0, sizeof(int) * ctx->att_count_elems, st) != cudaSuccess) return ESA_ERR_CUDA;
         return (esa_status)h;
     }
     return ESA_OK;
