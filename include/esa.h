@@ -33,8 +33,9 @@
  *     stream beside a select or attend of the same context, as long as the caller orders
  *     them against the calls that read the rows they write (the selection reads rows of M
  *     only, the attention reads every row up to the end of the current chunk).
- *   - Device-side problems (a bounded wait that ran out) are recorded in a status word
- *     read by esa_last_device_status; kernels never trap.
+ *   - Device-side problems (a bounded wait that ran out, a selected position outside the
+ *     middle tokens) are recorded in a status word read by esa_last_device_status; kernels
+ *     never trap and never read outside the caches.
  *   - The compressed-key cache is caller memory with library-defined contents: row p of
  *     sequence b is k'_p (bf16, d_c values).  n_prev[b] is the only record of its length.
  */
@@ -58,7 +59,8 @@ typedef enum {
     ESA_ERR_CUDA = 4,         /* a CUDA runtime call failed                           */
     ESA_ERR_TIMEOUT = 5,      /* a bounded device-side wait ran out                   */
     ESA_ERR_UNSUPPORTED = 6,  /* valid request the library does not implement         */
-    ESA_ERR_STATE = 7         /* call order: compressors not set                      */
+    ESA_ERR_STATE = 7,        /* call order: compressors not set                      */
+    ESA_ERR_INDEX = 8         /* a selected position passed to esa_attend lay outside M */
 } esa_status;
 
 /* Hyper-parameters of the step (paper symbols in comments) and capacities. */
@@ -131,7 +133,9 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
 /* Eq. 1 / Algorithm 1.  Q_cur: device [B, l_C, H, d].  K_cache, V_cache: device
  * [B, max_tokens, H_G, d] that already hold C at rows [n_prev[b], n_prev[b]+l_C).
  * idx: device int32 [B, top_k] and n_sel: device int32 [B] as written by esa_select
- * (positions must lie in M, ascending order is not required).  O: device [B, l_C, H, d]
+ * (positions must lie in M, ascending order is not required; a position outside M is
+ * replaced by the nearest position of M, so that no row outside the caches is read, and
+ * ESA_ERR_INDEX is recorded in the device status word).  O: device [B, l_C, H, d]
  * bf16.  Query head h reads key/value head h / (H/H_G).  Query c of the chunk attends
  * every I, selected-M and L key and the keys of C at chunk offsets <= c; bf16 products,
  * fp32 softmax and accumulation. */
@@ -161,7 +165,8 @@ esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
  * esa_attend_async; work is only enqueued on `stream`.
  *
  * The first call on each device looks up the array's device address; make that call with
- * the device current and before any stream capture is started on that device.  Every call
+ * the device current and before any stream capture is started on that device.  Host threads
+ * may make that first call at the same time (the look-up is serialised inside the library).  Every call
  * on a device shares the one array: calls that may overlap on the GPU (different streams,
  * no ordering between them) race on it and give wrong results; order them.  Nothing in the
  * array has to be cleared between calls -- each call writes every slot it later reads. */
@@ -174,6 +179,32 @@ esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const void* Q_cu
  * call.  Synchronises the given stream.  ESA_ERR_STATE if that call did no scoring. */
 esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int64_t n,
                                   void* stream);
+
+/* Diagnostic: copies q' (Eq. 5) of the most recent esa_select that scored -- its B * l_C
+ * rows of d_c bf16 values, row b * l_C + c for query c of sequence b -- to host memory
+ * dst_host[0 .. n_rows * d_c) as raw bf16 bit patterns.  Synchronises the given stream.
+ * ESA_ERR_STATE if that call did no scoring, ESA_ERR_CAPACITY if n_rows exceeds its rows. */
+esa_status esa_read_compressed_queries(esa_ctx* ctx, void* dst_host, int64_t n_rows, void* stream);
+
+/* Diagnostic of the bounded device-side waits: enqueues a one-thread kernel that waits, for
+ * at most limit_cycles SM clock cycles (1 <= limit_cycles <= 2e9, about a second), on a
+ * barrier that nothing ever completes.  The wait gives up, ESA_ERR_TIMEOUT is recorded in the
+ * status word and the kernel returns: the same path a kernel of the library takes when one of
+ * its waits runs out.  Nothing faults and the context stays usable. */
+esa_status esa_debug_wait_timeout(esa_ctx* ctx, int64_t limit_cycles, void* stream);
+
+/* Per-kernel timing.  While profiling is on, every kernel the context launches is bracketed by
+ * two CUDA events on the launching stream (events are created on first use and reused).  An
+ * event between two kernels of a step prevents the second from starting under the first one's
+ * tail, so profiled calls run somewhat slower than unprofiled ones: switch it on for sampled
+ * calls only.  esa_read_profile waits for the recorded events, adds the elapsed times up per
+ * kernel class (esa_kernel_class_count classes, named by esa_kernel_class_name; a class that
+ * covers two launches is timed across both) into launches[] / total_ms[] (n_classes entries,
+ * at least the class count) and forgets the records. */
+int32_t esa_kernel_class_count(void);
+const char* esa_kernel_class_name(int32_t cls);
+esa_status esa_set_profiling(esa_ctx* ctx, int32_t on);
+esa_status esa_read_profile(esa_ctx* ctx, int32_t n_classes, int64_t* launches, double* total_ms);
 
 /* Number of kernels this context has launched since creation (host counter). */
 int64_t esa_launch_count(const esa_ctx* ctx);

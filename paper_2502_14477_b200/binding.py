@@ -19,6 +19,7 @@ from .build import LIB_PATH
 STATUS_NAMES = {
     0: "ESA_OK", 1: "ESA_ERR_INVALID_ARG", 2: "ESA_ERR_SHAPE", 3: "ESA_ERR_CAPACITY",
     4: "ESA_ERR_CUDA", 5: "ESA_ERR_TIMEOUT", 6: "ESA_ERR_UNSUPPORTED", 7: "ESA_ERR_STATE",
+    8: "ESA_ERR_INDEX",
 }
 
 
@@ -84,6 +85,12 @@ _PROTOS = {
     "esa_attend_noalloc": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_read_pooled_scores": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
+    "esa_read_compressed_queries": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "esa_debug_wait_timeout": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
+    "esa_kernel_class_count": (C.c_int32, []),
+    "esa_kernel_class_name": (C.c_char_p, [C.c_int32]),
+    "esa_set_profiling": (C.c_int, [C.c_void_p, C.c_int32]),
+    "esa_read_profile": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "esa_launch_count": (C.c_int64, [C.c_void_p]),
     "esa_last_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
 }
@@ -278,6 +285,35 @@ class Esa:
         if st != 0:
             raise EsaError(st, "esa_read_pooled_scores")
         return out
+
+
+    def read_compressed_queries(self, n_rows: int, stream=None) -> np.ndarray:
+        """q' of the last scoring selection as bf16 bit patterns, uint16 [n_rows, d_c]."""
+        out = np.empty((n_rows, self.cfg.d_c), dtype=np.uint16)
+        st = self.lib.esa_read_compressed_queries(self._h, out.ctypes.data_as(C.c_void_p), n_rows, _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_read_compressed_queries")
+        return out
+
+    def set_profiling(self, on: bool):
+        st = self.lib.esa_set_profiling(self._h, 1 if on else 0)
+        if st != 0:
+            raise EsaError(st, "esa_set_profiling")
+
+    def read_profile(self) -> dict:
+        """{kernel class name: (launches, total ms)} of the launches profiled since the last read."""
+        n = int(self.lib.esa_kernel_class_count())
+        cnt = (C.c_int64 * n)()
+        ms = (C.c_double * n)()
+        st = self.lib.esa_read_profile(self._h, n, cnt, ms)
+        if st != 0:
+            raise EsaError(st, "esa_read_profile")
+        return {self.lib.esa_kernel_class_name(i).decode(): (int(cnt[i]), float(ms[i])) for i in range(n) if cnt[i]}
+
+    def debug_wait_timeout(self, limit_cycles: int, stream=None):
+        st = self.lib.esa_debug_wait_timeout(self._h, int(limit_cycles), _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_debug_wait_timeout")
 
 
 def attend_noalloc(cfg: EsaConfig, Q_cur, K_cache, V_cache, n_prev, idx, n_sel, O, stream=None):

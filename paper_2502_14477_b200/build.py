@@ -40,7 +40,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB_PATH
     cmd = [
-        _nvcc(), "-shared", "-Xcompiler", "-fPIC", "-std=c++17", "-O3", "-lineinfo",
+        _nvcc(), "-shared", "-Xcompiler", "-fPIC", "-std=c++17", "-O3", "-lineinfo", "--threads", "8",
         "-gencode", "arch=compute_100a,code=sm_100a",
         "-I", INCLUDE_DIR, "-I", CSRC,
         "-o", LIB_PATH,

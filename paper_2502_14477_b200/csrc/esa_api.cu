@@ -29,8 +29,8 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, ghist0, att, att_count, status, total;
-    size_t att_elems, att_count_elems;
+    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, ghist0, cidx, slice_cnt, ticket, att, att_count, status, total;
+    size_t att_elems, att_count_elems, slice_stride;
 };
 
 Layout make_layout(const esa_config* c) {
@@ -47,6 +47,10 @@ Layout make_layout(const esa_config* c) {
     L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.ghist0 = take(4 * (size_t)c->max_batch * 2048);
+    L.cidx = take(4 * (size_t)c->max_batch * c->max_tokens);
+    L.slice_stride = ((size_t)c->max_tokens + 4095) / 4096;
+    L.slice_cnt = take(4 * (size_t)c->max_batch * L.slice_stride);
+    L.ticket = take(4 * (size_t)c->max_batch);
     const size_t G = c->n_q_heads / c->n_kv_heads;
     size_t rows = (size_t)c->max_chunk * G;
     if (rows > (size_t)kAttSplitRows) rows = kAttSplitRows;
@@ -114,6 +118,7 @@ const char* esa_status_string(esa_status s) {
         case ESA_ERR_TIMEOUT: return "ESA_ERR_TIMEOUT";
         case ESA_ERR_UNSUPPORTED: return "ESA_ERR_UNSUPPORTED";
         case ESA_ERR_STATE: return "ESA_ERR_STATE";
+        case ESA_ERR_INDEX: return "ESA_ERR_INDEX";
     }
     return "ESA_ERR_UNKNOWN";
 }
@@ -138,6 +143,8 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->has_wmaps = false;
     c->launches = 0;
     c->last_scored = false;
+    c->last_q_rows = 0;
+    c->prof_on = false;
     if (cudaGetDevice(&c->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) {
         delete c;
@@ -161,6 +168,10 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
     c->ghist0 = reinterpret_cast<uint32_t*>(base + L.ghist0);
+    c->cidx = reinterpret_cast<int32_t*>(base + L.cidx);
+    c->sel_slice_cnt = reinterpret_cast<int*>(base + L.slice_cnt);
+    c->sel_ticket = reinterpret_cast<int*>(base + L.ticket);
+    c->sel_slice_stride = (int)L.slice_stride;
     c->last_decode = false;
     c->att_part = reinterpret_cast<float*>(base + L.att);
     c->att_part_elems = L.att_elems;
@@ -168,6 +179,7 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->att_count_elems = L.att_count_elems;
     c->status = reinterpret_cast<int*>(base + L.status);
     if (cudaMemset(c->status, 0, 256) != cudaSuccess ||
+        cudaMemset(c->sel_ticket, 0, 4 * (size_t)cfg->max_batch) != cudaSuccess ||
         cudaMemset(c->att_count, 0, 4 * L.att_count_elems) != cudaSuccess) {
         cudaFree(base);
         delete c;
@@ -179,6 +191,11 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
 
 esa_status esa_destroy(esa_ctx* ctx) {
     if (!ctx) return ESA_ERR_INVALID_ARG;
+    for (auto& r : ctx->prof_recs) {
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    for (auto ev : ctx->prof_pool) cudaEventDestroy(ev);
     cudaError_t e = cudaFree(ctx->base);
     delete ctx;
     return from_cuda(e);
@@ -291,6 +308,7 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
         if (lM > ctx->cfg.top_k) any_large = true; else any_small = true;
     }
     ctx->last_scored = any_large;
+    ctx->last_q_rows = any_large ? (int64_t)B * l_C : 0;
     cudaError_t e = cudaSuccess;
     if (any_small) {
         e = launch_select_all(ctx, B, meta, idx_out, n_sel_out, st);
@@ -327,9 +345,11 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     for (int b = 0; b < B; ++b)
         if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
     ctx->last_decode = l_C == 1;
-    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, ghist_cleared, st);
+    bool pooled_ready = false;
+    e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, ghist_cleared, st,
+                     &pooled_ready);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
-    e = launch_select(ctx, B, l_C, smeta, max_lM, idx_out, n_sel_out, st);
+    e = launch_select(ctx, B, l_C, smeta, max_lM, pooled_ready, idx_out, n_sel_out, st);
     return from_cuda(e);
 }
 
@@ -371,11 +391,67 @@ esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int6
     if (n > ctx->last_lM[b]) return ESA_ERR_CAPACITY;
     if (n == 0) return ESA_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    // the aggregated-score buffer of this sequence is free again after the selection: stage there
+    // the candidate-key buffer of this sequence is free again after the selection: stage there
     float* tmp = reinterpret_cast<float*>(ctx->skey + (int64_t)b * ctx->cfg.max_tokens);
     if (launch_read_pooled(ctx, b, tmp, n, st) != cudaSuccess) return ESA_ERR_CUDA;
     if (cudaMemcpyAsync(dst_host, tmp, 4 * (size_t)n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ESA_ERR_CUDA;
     return from_cuda(cudaStreamSynchronize(st));
+}
+
+esa_status esa_read_compressed_queries(esa_ctx* ctx, void* dst_host, int64_t n_rows, void* stream) {
+    if (!ctx || !dst_host || n_rows < 0) return ESA_ERR_INVALID_ARG;
+    if (!ctx->last_scored || ctx->last_q_rows == 0) return ESA_ERR_STATE;
+    if (n_rows > ctx->last_q_rows) return ESA_ERR_CAPACITY;
+    if (n_rows == 0) return ESA_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(dst_host, ctx->Qc, 2 * (size_t)n_rows * ctx->dc, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ESA_ERR_CUDA;
+    return from_cuda(cudaStreamSynchronize(st));
+}
+
+esa_status esa_debug_wait_timeout(esa_ctx* ctx, int64_t limit_cycles, void* stream) {
+    if (!ctx || limit_cycles < 1 || limit_cycles > 2000000000LL) return ESA_ERR_INVALID_ARG;
+    return from_cuda(launch_debug_wait(ctx, limit_cycles, (cudaStream_t)stream));
+}
+
+int32_t esa_kernel_class_count(void) { return KC_COUNT; }
+
+const char* esa_kernel_class_name(int32_t cls) {
+    static const char* names[KC_COUNT] = {
+        "compress_tc_kernel", "compress_gemv_kernel", "compress_kernel", "append_kv_kernel", "score_tc_kernel<.,1>",
+        "score_tc_kernel<.,2>", "score_pass_kernel<.,1>+<.,2>", "score_decode_kernel", "pool_hist_kernel",
+        "select_topk_kernel", "select_all_kernel", "attend_tc_kernel", "attend_decode_kernel", "attend_kernel",
+        "attend_merge_kernel"};
+    return cls >= 0 && cls < KC_COUNT ? names[cls] : "";
+}
+
+esa_status esa_set_profiling(esa_ctx* ctx, int32_t on) {
+    if (!ctx) return ESA_ERR_INVALID_ARG;
+    ctx->prof_on = on != 0;
+    return ESA_OK;
+}
+
+esa_status esa_read_profile(esa_ctx* ctx, int32_t n_classes, int64_t* launches, double* total_ms) {
+    if (!ctx || !launches || !total_ms || n_classes < KC_COUNT) return ESA_ERR_INVALID_ARG;
+    for (int i = 0; i < n_classes; ++i) {
+        launches[i] = 0;
+        total_ms[i] = 0.0;
+    }
+    esa_status result = ESA_OK;
+    for (auto& r : ctx->prof_recs) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) {
+            cudaGetLastError();
+            result = ESA_ERR_CUDA;
+        } else {
+            launches[r.cls] += 1;
+            total_ms[r.cls] += ms;
+        }
+        ctx->prof_pool.push_back(r.a);
+        ctx->prof_pool.push_back(r.b);
+    }
+    ctx->prof_recs.clear();
+    return result;
 }
 
 int64_t esa_launch_count(const esa_ctx* ctx) { return ctx ? ctx->launches : -1; }
@@ -390,6 +466,7 @@ esa_status esa_last_device_status(esa_ctx* ctx, void* stream) {
         if (cudaMemsetAsync(ctx->status, 0, sizeof(int), st) != cudaSuccess) return ESA_ERR_CUDA;
         // a kernel that gave up may have left arrival counters of the in-kernel merges behind
         if (cudaMemsetAsync(ctx->att_count, 0, sizeof(int) * ctx->att_count_elems, st) != cudaSuccess) return ESA_ERR_CUDA;
+        if (cudaMemsetAsync(ctx->sel_ticket, 0, sizeof(int) * ctx->cfg.max_batch, st) != cudaSuccess) return ESA_ERR_CUDA;
         return (esa_status)h;
     }
     return ESA_OK;

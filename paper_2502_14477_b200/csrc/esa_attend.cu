@@ -20,6 +20,8 @@
 // sequence), the kernel that merges the partial (O, m, l) triples of key-list splits -- the
 // same algebra as Algorithm 1's merge -- and the entry point that needs no allocation.
 // Prefill-sized chunks run in esa_attend_tc.cu.
+#include <mutex>
+
 #include "esa_internal.h"
 
 namespace esa {
@@ -33,6 +35,7 @@ struct AttendParams {
     const int32_t* n_sel;     // [B]
     float* part;              // split partials
     int* unit_count;          // arrival counters per (sequence, key/value head) for the in-kernel merge of the decode kernel
+    int* status;              // device status word (may be null: the entry point without a context)
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
@@ -82,6 +85,7 @@ attend_kernel(AttendParams p) {
     const int32_t* idx = p.idx + (int64_t)b * p.top_k;
     const int64_t tok_stride = (int64_t)p.HG * D;
 
+    int bad_idx = 0;
     auto load_kv = [&](int st, int tile) {
         uint4* dk = sK + st * BN * CH;
         uint4* dv = sV + st * BN * CH;
@@ -92,7 +96,7 @@ attend_kernel(AttendParams p) {
             int pos = 0;
             if (ok) {
                 if (j < i_end) pos = j;
-                else if (j < n_glob) pos = __ldg(idx + (j - i_end));
+                else if (j < n_glob) pos = clamp_selected(__ldg(idx + (j - i_end)), i_end, m_end, bad_idx);
                 else pos = m_end + (j - n_glob);
             }
             const int64_t off = (int64_t)pos * tok_stride + c * 8;
@@ -229,6 +233,7 @@ attend_kernel(AttendParams p) {
         __syncthreads();
     }
     cp_async_wait<0>();
+    if (bad_idx && p.status) atomicExch(p.status, kStatusBadIndex);
 
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
@@ -373,6 +378,7 @@ attend_decode_kernel(AttendParams p) {
     const int64_t tok_stride = (int64_t)p.HG * D;
 
     // list positions -> token positions of the rows of iteration `it` that this lane copies
+    int bad_idx = 0;
     auto lookup = [&](int it, int (&pos)[PER_LANE]) {
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) {
@@ -380,7 +386,7 @@ attend_decode_kernel(AttendParams p) {
             int q = -1;
             if (it < it_end && j < n_att) {
                 if (j < i_end) q = j;
-                else if (j < n_glob) q = __ldg(idx + (j - i_end));
+                else if (j < n_glob) q = clamp_selected(__ldg(idx + (j - i_end)), i_end, m_end, bad_idx);
                 else q = m_end + (j - n_glob);
             }
             pos[i] = q;
@@ -498,6 +504,7 @@ attend_decode_kernel(AttendParams p) {
         __syncwarp();          // the stage is free for the copy issued next iteration
     }
     cp_async_wait<0>();
+    if (bad_idx && p.status) atomicExch(p.status, kStatusBadIndex);
 
     // the lanes that share a head pair (same lane & 3) each saw different rows: add their sums
 #pragma unroll
@@ -590,6 +597,7 @@ static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     p.nsplit = nsplit;
     if ((size_t)B * p.HG > ctx->att_count_elems) return cudaErrorInvalidConfiguration;
     p.unit_count = ctx->att_count;
+    ProfScope prof(ctx, KC_ATTEND_DECODE, st);
     e = launch_pdl(attend_decode_kernel<D, G>, dim3(nsplit, p.HG, B), dim3(DEC_WARPS * 32), smem, st, p);
     ctx->launches += 1;
     return e;
@@ -630,9 +638,13 @@ static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
         if (nsplit < 1) nsplit = 1;
     }
     p.nsplit = nsplit;
-    attend_kernel<D, NW, BN><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
+    {
+        ProfScope prof(ctx, KC_ATTEND_SMALL, st);
+        attend_kernel<D, NW, BN><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
+    }
     ctx->launches += 1;
     if (nsplit > 1) {
+        ProfScope prof(ctx, KC_ATTEND_MERGE, st);
         attend_merge_kernel<D><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
         ctx->launches += 1;
     }
@@ -644,6 +656,7 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
                           const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st) {
     AttendParams p;
     p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
+    p.status = ctx->status;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
@@ -699,6 +712,7 @@ struct NoAllocDevice {
     bool ready;
 };
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;      // host threads may make a device's first call together
 
 template <int D, int NW, int BN>
 cudaError_t launch_noalloc_t(const NoAllocDevice& dev, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
@@ -763,6 +777,7 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess) return ESA_ERR_CUDA;
     if (device < 0 || device >= kNoAllocMaxDevices) return ESA_ERR_UNSUPPORTED;
+    std::unique_lock<std::mutex> lock(g_noalloc_mutex);
     NoAllocDevice& dev = g_noalloc_dev[device];
     if (!dev.ready) {
         void* ptr = nullptr;
@@ -777,10 +792,11 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
         dev.num_sms = sms;
         dev.ready = true;
     }
+    lock.unlock();
 
     AttendParams p;
     p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
-    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr;
+    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr;
     p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
     p.top_k = cfg->top_k; p.nsplit = 1;
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)D);

@@ -559,6 +559,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
         const uint32_t blk_off = (chunk >> 3) * KV_BLK_BYTES;
+        int bad_idx = 0;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % TC_STAGES;
             const uint32_t ph = ((j / TC_STAGES) & 1) ^ 1;
@@ -569,7 +570,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 const int jj = key0 + rsub + it * RSTEP;
                 int q = -1;
                 if (jj < i_end) q = jj;
-                else if (jj < n_glob) q = __ldg(idx + (jj - i_end));
+                else if (jj < n_glob) q = clamp_selected(__ldg(idx + (jj - i_end)), i_end, m_end, bad_idx);
                 else if (jj < n_att) q = m_end + (jj - n_glob);
                 pos[it] = q;
             }
@@ -590,6 +591,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             }
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
         }
+        if (bad_idx) atomicExch(p.status, kStatusBadIndex);
         cp_async_wait<0>();
     } else if (warp_u < TC_MMA_WARP + 2 && n_tiles > 0) {
         // ------------------------------------------------------------ MMA issue: one converged warp per Q tile,
@@ -691,6 +693,7 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     CUtensorMap qmap;
     p.q_tma = make_tensor_map_q(&qmap, p.Q, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
     if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
+    ProfScope prof(ctx, KC_ATTEND_TC, st);
     e = launch_pdl(attend_tc_kernel<D>, dim3(row_tiles, p.HG, B * best), dim3(TC_THREADS), smem, st, qmap, p);
     ctx->launches += 1;
     return e;

@@ -46,6 +46,18 @@ __device__ __forceinline__ int swz(int row, int chunk) {
     }
 }
 
+// A selected position handed to the attention must lie in M = [i_end, m_end).  One that does not
+// (a stale or corrupted index buffer) is replaced by the nearest position of M, so that no row
+// outside the caches is ever read, and `bad` is raised; the caller records ESA_ERR_INDEX once.
+constexpr int kStatusBadIndex = 8;
+__device__ __forceinline__ int clamp_selected(int q, int i_end, int m_end, int& bad) {
+    if ((unsigned)(q - i_end) >= (unsigned)(m_end - i_end)) {
+        bad = 1;
+        q = q < i_end ? i_end : m_end - 1;
+    }
+    return q;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

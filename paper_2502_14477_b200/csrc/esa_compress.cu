@@ -149,6 +149,7 @@ static cudaError_t launch_compress_t(esa_ctx* ctx, const __nv_bfloat16* X, int r
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    ProfScope prof(ctx, KC_COMPRESS_MMA, st);
     e = cudaLaunchKernelEx(&cfg, compress_kernel<DC>, X, W, bias, dst, rows, rows_per_seq, d_in, kslice,
                            seq_stride, map);
     ctx->launches += 1;
@@ -243,6 +244,7 @@ cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, in
     const int rows = B * rows_per_seq;
     if (rows > kCompressGemvRows || d_in % 8 != 0) return cudaErrorNotSupported;
     const dim3 grid(ctx->dc, (rows + GEMV_ROWS - 1) / GEMV_ROWS);
+    ProfScope prof(ctx, KC_COMPRESS_GEMV, st);
     cudaError_t e = launch_pdl(compress_gemv_kernel, grid, dim3(GEMV_THREADS), 0, st, X, W, bias, dst, rows,
                                rows_per_seq, d_in, ctx->dc, dst_seq_stride, map, zero_words, zero_count, zero2_words,
                                zero2_count);
@@ -277,6 +279,7 @@ cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new, co
     int gx = (int)((per_seq + 255) / 256);
     if (gx > 4 * ctx->num_sms) gx = 4 * ctx->num_sms;
     if (gx < 1) gx = 1;
+    ProfScope prof(ctx, KC_APPEND_KV, st);
     cudaError_t e = launch_pdl(append_kv_kernel, dim3(gx, B), dim3(256), 0, st,
                                reinterpret_cast<const uint4*>(K_new), reinterpret_cast<const uint4*>(V_new),
                                reinterpret_cast<uint4*>(K_cache), reinterpret_cast<uint4*>(V_cache), n_new, row_chunks,

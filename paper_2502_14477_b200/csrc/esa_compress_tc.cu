@@ -231,6 +231,7 @@ cudaError_t launch_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_pe
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
+    ProfScope prof(ctx, KC_COMPRESS_TC, st);
     e = cudaLaunchKernelEx(&cfg, compress_tc_kernel<DC>, xmap, *wmap, p);
     ctx->launches += 1;
     return e;

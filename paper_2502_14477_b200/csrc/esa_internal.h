@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/esa.h"
 #include "esa_common.cuh"
 
@@ -40,6 +42,17 @@ struct RowMap {
     int row0[kMaxBatch];
 };
 
+// Kernel classes of the per-kernel timing facility (esa_set_profiling / esa_read_profile).
+enum KernelClass {
+    KC_COMPRESS_TC = 0, KC_COMPRESS_GEMV, KC_COMPRESS_MMA, KC_APPEND_KV, KC_SCORE_PASS1, KC_SCORE_PASS2, KC_SCORE_MMA,
+    KC_SCORE_DECODE, KC_POOL_HIST, KC_SELECT_TOPK, KC_SELECT_ALL, KC_ATTEND_TC, KC_ATTEND_DECODE, KC_ATTEND_SMALL,
+    KC_ATTEND_MERGE, KC_COUNT
+};
+struct ProfRec {
+    int cls;
+    cudaEvent_t a, b;
+};
+
 }  // namespace esa
 
 struct esa_ctx {
@@ -58,9 +71,14 @@ struct esa_ctx {
     float* bk;           // [dc]
     __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
     uint32_t* rkey;      // [max_batch * max_chunk] ordered keys of the row maxima r_c
-    uint32_t* skey;      // [max_batch, max_tokens] aggregated scores (ordered keys); unused when l_C = 1
+    uint32_t* skey;      // [max_batch, max_tokens] unpooled aggregated scores (ordered keys) of the scoring paths that do not pool;
+                         // afterwards the selection's candidate keys
     uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys (l_C = 1: of the pooled raw scores, r not yet subtracted)
-    uint32_t* ghist0;    // [max_batch, 2048] first-digit histograms of pkey, filled by the decode scoring kernel
+    uint32_t* ghist0;    // [max_batch, 2048] histograms of pkey's top 11 bits (first radix digit)
+    int32_t* cidx;       // [max_batch, max_tokens] positions of the selection's candidates
+    int* sel_slice_cnt;  // [max_batch, sel_slice_stride] candidates per 4096-token slice
+    int* sel_ticket;     // [max_batch] arrival tickets of the selection kernel; 0 between launches
+    int sel_slice_stride;
     bool last_decode;    // the last selection ran with l_C = 1 (pkey holds raw pooled scores)
     float* att_part;     // split-KV partial outputs + (m, l)
     size_t att_part_elems;
@@ -70,10 +88,43 @@ struct esa_ctx {
     int64_t launches;
     int last_lM[esa::kMaxBatch];
     bool last_scored;
+    int64_t last_q_rows;  // rows of q' left in Qc by the last selection that scored
     size_t ws_bytes;
+    bool prof_on;                          // bracket every kernel launch with CUDA events
+    std::vector<esa::ProfRec> prof_recs;   // launches recorded since the last esa_read_profile
+    std::vector<cudaEvent_t> prof_pool;    // events free for reuse
 };
 
 namespace esa {
+
+// While profiling is on, records a CUDA event on the launching stream before and after the kernel(s)
+// launched during its lifetime (class `cls`).  An event between two kernels keeps the second from being
+// set up under the first one's tail, so profiled calls run without the dependent-launch overlap.
+struct ProfScope {
+    esa_ctx* c;
+    cudaStream_t st;
+    cudaEvent_t b;
+    bool on;
+    ProfScope(esa_ctx* ctx, int cls, cudaStream_t stream) : c(ctx), st(stream), b(nullptr), on(ctx->prof_on) {
+        if (!on) return;
+        cudaEvent_t ev[2] = {nullptr, nullptr};
+        for (int i = 0; i < 2; ++i) {
+            if (!c->prof_pool.empty()) {
+                ev[i] = c->prof_pool.back();
+                c->prof_pool.pop_back();
+            } else if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+                on = false;
+                return;
+            }
+        }
+        cudaEventRecord(ev[0], st);
+        b = ev[1];
+        c->prof_recs.push_back(ProfRec{cls, ev[0], ev[1]});
+    }
+    ~ProfScope() {
+        if (on) cudaEventRecord(b, st);
+    }
+};
 
 // Y[dst rows] = bf16( X[rows, d_in] . W[dc, d_in]^T + bias ), fp32 accumulation, split-K.
 cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
@@ -83,16 +134,19 @@ cudaError_t launch_compress(esa_ctx* ctx, const __nv_bfloat16* X, int B, int row
 // Eq. 6 + Eq. 4: fills ctx->skey (and ctx->rkey) for the middle tokens of every sequence.
 // l_C = 1: fills ctx->pkey (pooled raw scores), ctx->ghist0 and ctx->rkey instead.
 // rkey_cleared / ghist_cleared: the caller's compression kernel has already zeroed ctx->rkey / ctx->ghist0 for this call.
+// *pooled_ready: ctx->pkey and ctx->ghist0 hold the pooled keys and their first-digit histogram; otherwise
+// ctx->skey holds unpooled keys and ctx->ghist0 is zero.
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                         const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st);
+                         const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st,
+                         bool* pooled_ready);
 
 // The same for chunks of >= 64 queries and d' in {64, 128} on tcgen05 with TMA-fed tiles; expects
-// ctx->rkey zeroed (pass 1 clears the part of ctx->skey that pass 2 accumulates into).  cudaErrorNotSupported when the shape is not covered.
+// ctx->rkey zeroed (pass 1 clears what pass 2 accumulates into).  cudaErrorNotSupported when the shape is not covered.
 cudaError_t launch_score_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                            const SeqMeta& meta, int max_lM, cudaStream_t st);
+                            const SeqMeta& meta, int max_lM, cudaStream_t st, bool* pooled_ready);
 
-// Eq. 8 + Eq. 2 on ctx->skey -> idx_out / n_sel_out.
-cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM,
+// Eq. 8 (unless pooled_ready) + Eq. 2 -> idx_out / n_sel_out.
+cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, bool pooled_ready,
                           int32_t* idx_out, int32_t* n_sel_out, cudaStream_t st);
 
 // idx_out[b, 0..l_M) = i_end + 0..l_M-1, n_sel_out[b] = l_M for sequences with l_M <= top_k
@@ -145,5 +199,8 @@ cudaError_t launch_append_kv(esa_ctx* ctx, int B, const __nv_bfloat16* K_new,
                              __nv_bfloat16* V_cache, const RowMap& map, cudaStream_t st);
 
 cudaError_t launch_read_pooled(esa_ctx* ctx, int b, float* dst_dev, int64_t n, cudaStream_t st);
+
+// One thread waits on a barrier nobody completes, for at most limit_cycles: exercises the give-up path.
+cudaError_t launch_debug_wait(esa_ctx* ctx, int64_t limit_cycles, cudaStream_t st);
 
 }  // namespace esa

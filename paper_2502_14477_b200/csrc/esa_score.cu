@@ -320,8 +320,10 @@ score_decode_kernel(ScoreDecodeParams p) {
 
 template <int DC>
 static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
-                                  const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st) {
+                                  const SeqMeta& meta, int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st,
+                                  bool* pooled_ready) {
     cudaError_t e = cudaSuccess;
+    *pooled_ready = false;
     if (!rkey_cleared) e = cudaMemsetAsync(ctx->rkey, 0, sizeof(uint32_t) * (size_t)B * l_C, st);
     if (e != cudaSuccess) return e;
     if (l_C == 1) {
@@ -344,16 +346,21 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
         p.chunk = (int)chunk;
         int gx = (max_lM + p.chunk - 1) / p.chunk;
         if (gx < 1) gx = 1;
+        ProfScope prof(ctx, KC_SCORE_DECODE, st);
         e = launch_pdl(score_decode_kernel<DC>, dim3(gx, B), dim3(SD_THREADS), 0, st, p);
         ctx->launches += 1;
+        *pooled_ready = true;
         return e;
     }
-    // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels (they clear skey themselves)
+    // prefill-sized chunks with d' of 64 or 128: tcgen05 + TMA kernels (they clear what they accumulate into)
     if (score_uses_tc(ctx, B, l_C)) {
-        e = launch_score_tc(ctx, B, l_C, kc_cache, meta, max_lM, st);
+        e = launch_score_tc(ctx, B, l_C, kc_cache, meta, max_lM, st, pooled_ready);
         if (e != cudaErrorNotSupported) return e;
         cudaGetLastError();
     }
+    // the pooling kernel that follows adds to the first-digit histograms
+    e = cudaMemsetAsync(ctx->ghist0, 0, sizeof(uint32_t) * (size_t)B * SD_BINS, st);
+    if (e != cudaSuccess) return e;
     e = cudaMemset2DAsync(ctx->skey, sizeof(uint32_t) * ctx->cfg.max_tokens, 0,
                           sizeof(uint32_t) * (size_t)max_lM, B, st);
     if (e != cudaSuccess) return e;
@@ -371,6 +378,7 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
     e = cudaFuncSetAttribute(score_pass_kernel<DC, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(gx, qblocks, B);
+    ProfScope prof(ctx, KC_SCORE_MMA, st);
     score_pass_kernel<DC, 1><<<grid, SC_THREADS, smem, st>>>(p);
     score_pass_kernel<DC, 2><<<grid, SC_THREADS, smem, st>>>(p);
     ctx->launches += 2;
@@ -378,11 +386,11 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
 }
 
 cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache, const SeqMeta& meta,
-                         int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st) {
+                         int max_lM, bool rkey_cleared, bool ghist_cleared, cudaStream_t st, bool* pooled_ready) {
     switch (ctx->dc) {
-        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
-        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
-        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st);
+        case 32: return launch_score_t<32>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st, pooled_ready);
+        case 64: return launch_score_t<64>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st, pooled_ready);
+        case 128: return launch_score_t<128>(ctx, B, l_C, kc_cache, meta, max_lM, rkey_cleared, ghist_cleared, st, pooled_ready);
     }
     return cudaErrorInvalidValue;
 }

@@ -69,11 +69,12 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
 // ESA_ERR_TIMEOUT (5) in the device status word and raises the CTA-wide abort flag; from
 // then on every wait of the CTA returns at once, so the kernel drains, frees its tensor
 // memory and exits with wrong data but a usable context.
+constexpr long long kWaitLimitCycles = 4000000000LL;
 struct WaitCtx {
     volatile int* abort_flag;   // shared memory
     int* status;                // global status word
+    long long limit = kWaitLimitCycles;   // SM clock cycles after which a wait gives up
 };
-constexpr long long kWaitLimitCycles = 4000000000LL;
 constexpr uint32_t kParkNs = 20000;     // one parked try_wait lasts at most this long
 
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
@@ -82,7 +83,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
     while (true) {
         if (mbar_try_wait_parked(bar, parity, kParkNs)) return;
         if (*w.abort_flag) return;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > w.limit) {
             *w.abort_flag = 1;
             atomicExch(w.status, 5);
             return;
