@@ -88,6 +88,61 @@ def score_flops(cfg, t: int, l_C: int) -> float:
     return (2.0 * cfg.d_c + 1.0) * l_C * l_M if l_M > cfg.k else 0.0
 
 
+def partition_sizes(cfg, t: int, l_C: int):
+    i_end = min(cfg.l_I, t)
+    m_end = max(i_end, t - cfg.l_L)
+    l_M = m_end - i_end
+    return i_end, l_M, i_end + min(cfg.k, l_M) + (t - m_end) + l_C
+
+
+def compress_flops(cfg, l_C: int) -> float:
+    """Eq. 5 for the chunk's keys and queries: 2 l_C d' (d_H + d_G)."""
+    return 2.0 * l_C * cfg.d_c * (cfg.d_H + cfg.d_G)
+
+
+def select_bytes(cfg, t: int, l_C: int) -> float:
+    """Eq. 2: read 4 l_M, write 4 k (only when l_M > k)."""
+    _, l_M, _ = partition_sizes(cfg, t, l_C)
+    return 4.0 * l_M + 4.0 * cfg.k if l_M > cfg.k else 0.0
+
+
+def kernel_rooflines(prof: dict, sampled, cfg, peaks):
+    """Per-kernel achieved rates of the profiled chunks: algorithmic work of those chunks / summed
+    CUDA-event time of the kernel class, against the measured sustained and burst bf16 peaks
+    (contractions) or the measured copy bandwidth (selection)."""
+    sc = sum(score_flops(cfg, t, l_C) for t, l_C in sampled)
+    out = {}
+
+    def tensor(name, flops, note=None):
+        if name not in prof or prof[name][1] <= 0:
+            return
+        n, ms = prof[name]
+        tf = flops / (ms * 1e-3) / 1e12
+        out[name] = {"bound": "tensor", "launches": n, "us_per_launch": 1e3 * ms / n, "achieved": tf, "unit": "TFLOP/s",
+                     "frac_sustained": tf / peaks["tflops_sustained"], "frac_burst": tf / peaks["tflops_burst"]}
+        if note:
+            out[name]["note"] = note
+
+    tensor("attend_tc_kernel", sum(attend_flops(cfg, t, l_C) for t, l_C in sampled))
+    tensor("score_tc_kernel<.,1>", sc, "one pass: (2 d' + 1) l_C l_M flops per launch")
+    tensor("score_tc_kernel<.,2>", sc, "second pass over the same products (the method counts one), with Eq. 4, Eq. 8 and the first radix digit in the epilogue")
+    tensor("compress_tc_kernel", sum(compress_flops(cfg, l_C) for t, l_C in sampled),
+           "both compressions of a chunk (keys on the side stream, queries ahead of the scoring); latency-bound launches")
+    if "score_tc_kernel<.,1>" in out and "score_tc_kernel<.,2>" in out:
+        ms = prof["score_tc_kernel<.,1>"][1] + prof["score_tc_kernel<.,2>"][1]
+        tf = sc / (ms * 1e-3) / 1e12
+        out["scoring, both passes against the method's one-pass work"] = {
+            "bound": "tensor", "achieved": tf, "unit": "TFLOP/s", "frac_sustained": tf / peaks["tflops_sustained"],
+            "frac_burst": tf / peaks["tflops_burst"]}
+    if "select_topk_kernel" in prof and prof["select_topk_kernel"][1] > 0:
+        n, ms = prof["select_topk_kernel"]
+        gbs = sum(select_bytes(cfg, t, l_C) for t, l_C in sampled) / (ms * 1e-3) / 1e9
+        out["select_topk_kernel"] = {"bound": "latency", "launches": n, "us_per_launch": 1e3 * ms / n, "achieved": gbs,
+                                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                                     "note": "read 4 l_M + write 4 k bytes per launch: far too little to load HBM"}
+    return out
+
+
 def decode_bytes(cfg, t: int) -> float:
     """Algorithmic HBM bytes of one decode step of one sequence: 2 l_M d' + 4 n_att d_G."""
     i_end = min(cfg.l_I, t)
@@ -187,17 +242,18 @@ def _side_stream():
     return _SIDE[0]
 
 
-ATTEND_EVENT_EVERY = 8      # one attention launch in this many carries CUDA events (see run_prefill_layer)
+PROFILE_EVERY = 8      # one chunk in this many runs with per-kernel CUDA events (see run_prefill_layer)
 
 
-def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None, phase=0):
+def run_prefill_layer(ctx, cfg, L, bufs, sampled=None, phase=0):
     """The whole chunked prefill of one layer with inputs resident in HBM.
 
-    attend_events: list that receives (t, l_C, start, end) CUDA events around attention launches.
-    An event record between two kernels keeps the second one from being set up under the first
-    one's tail (programmatic dependent launch), which costs 8 % of the step when every launch is
-    bracketed; so one launch in ATTEND_EVENT_EVERY is, the sampled position rotating with `phase`
-    (over 8 steps every chunk position is sampled once)."""
+    sampled: list that receives (t, l_C) of the chunks whose kernels were individually timed.  On
+    such a chunk the library brackets every kernel with CUDA events on the launching stream
+    (esa_set_profiling).  An event record between two kernels keeps the second one from being set
+    up under the first one's tail (programmatic dependent launch), which costs 8 % of the step when
+    every launch is bracketed; so one chunk in PROFILE_EVERY is, the sampled position rotating with
+    `phase` (over 8 steps every chunk position is sampled once)."""
     Kc, idx, n_sel, O = bufs
     # The compressed keys of the current chunk are not read by this chunk's selection (C is not
     # part of M): esa_compress_keys runs on a side stream beside the attention, and the selection
@@ -209,6 +265,9 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None, phase=0):
     for t in range(0, cfg.S, cfg.l_C):
         l_C = min(cfg.l_C, cfg.S - t)
         Qc = L.Q[:, t: t + l_C]
+        timed = sampled is not None and (t // cfg.l_C + phase) % PROFILE_EVERY == 0
+        if timed:
+            ctx.set_profiling(True)
         with torch.cuda.stream(side):
             ctx.compress_keys(L.K[:, t: t + l_C], Kc, [t])
             ev = torch.cuda.Event()
@@ -222,14 +281,10 @@ def run_prefill_layer(ctx, cfg, L, bufs, attend_events=None, phase=0):
         if c_need >= 0 and not done[c_need].query():
             main.wait_event(done[c_need])
         ctx.select(Qc, Kc, [t], idx, n_sel)
-        timed = attend_events is not None and (t // cfg.l_C + phase) % ATTEND_EVENT_EVERY == 0
-        if timed:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
         ctx.attend(Qc, L.K, L.V, [t], idx, n_sel, O[:, t: t + l_C])
         if timed:
-            e1.record()
-            attend_events.append((t, l_C, e0, e1))
+            ctx.set_profiling(False)
+            sampled.append((t, l_C))
     main.wait_stream(side)
 
 
@@ -396,6 +451,14 @@ def time_decode(cfg3, n_steps, rank_seed):
     for i in range(min(8, n_steps)):
         step(i)
     torch.cuda.synchronize()
+    # per-kernel times of a few steps, outside the timed region (events between the kernels of a step
+    # keep each from starting under its predecessor's tail)
+    ctx.set_profiling(True)
+    for i in range(min(8, n_steps)):
+        step(i)
+    ctx.set_profiling(False)
+    torch.cuda.synchronize()
+    prof = {k: {"launches": n, "us_per_launch": 1e3 * ms / n} for k, (n, ms) in ctx.read_profile().items()}
     l0 = ctx.launch_count
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -409,7 +472,100 @@ def time_decode(cfg3, n_steps, rank_seed):
     launches = (ctx.launch_count - l0) / n_steps
     assert ctx.last_device_status() == 0
     ctx.close()
-    return us, byts, launches
+    return us, byts, launches, prof
+
+
+class DeviceLayer:
+    """Q/K/V of one layer drawn on the device (N(0,1) bf16, optional per-head scale U(0.5, 2)): the
+    secondary prefill legs use it to keep start-up short."""
+
+    def __init__(self, cfg, seed):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(seed)
+        mk = lambda nh: torch.randn(1, cfg.S, nh, cfg.d, device="cuda", dtype=torch.bfloat16, generator=g)
+        self.Q, self.K, self.V = mk(cfg.H), mk(cfg.H_G), mk(cfg.H_G)
+        if cfg.kind == "headscale":
+            for x in (self.Q, self.K, self.V):
+                x.mul_((0.5 + 1.5 * torch.rand(1, 1, x.shape[2], 1, device="cuda", generator=g)).to(torch.bfloat16))
+        self.wq, self.wk = syn.compressor_weights(cfg, 0)
+
+
+def time_prefill_leg(name, steps, peaks):
+    """Whole chunked prefill of one layer of a secondary workload (c2: 32k, c4: 256k in chunks of 1024)."""
+    cfg = syn.get_config(name)
+    L = DeviceLayer(cfg, cfg.seed)
+    ctx = make_ctx(cfg, cfg.S, cfg.l_C, 1)
+    ctx.set_compressors(L.wq, None, L.wk, None)
+    bufs = (torch.zeros(1, cfg.S, cfg.d_c, dtype=torch.bfloat16, device="cuda"),
+            torch.zeros(1, cfg.k, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda"),
+            torch.empty(1, cfg.S, cfg.H, cfg.d, dtype=torch.bfloat16, device="cuda"))
+    for i in range(2):
+        run_prefill_layer(ctx, cfg, L, bufs)
+    torch.cuda.synchronize()
+    ctx.read_profile()
+    sampled = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        run_prefill_layer(ctx, cfg, L, bufs, sampled, phase=i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert ctx.last_device_status() == 0
+    prof = ctx.read_profile()
+    by_kernel = kernel_rooflines(prof, sampled, cfg, peaks)
+    n_chunks = (cfg.S + cfg.l_C - 1) // cfg.l_C
+    att_ms = sum(v[1] for k, v in prof.items() if k.startswith("attend"))
+    out = {"workload": f"{name}: H={cfg.H} H_G={cfg.H_G} d={cfg.d} d'={cfg.d_c}, {cfg.S}-token prefill in chunks of {cfg.l_C}, "
+                       f"l_I={cfg.l_I} l_L={cfg.l_L} k={cfg.k} eps={cfg.eps}; inputs drawn on the device",
+           "ms_per_layer": ms, "tokens_per_s_per_layer": cfg.S / (ms * 1e-3), "steps": steps,
+           "attention_share_of_step": att_ms * (steps * n_chunks / max(1, len(sampled))) / (ms * steps),
+           "roofline_by_kernel": by_kernel}
+    ctx.close()
+    del L, bufs
+    torch.cuda.empty_cache()
+    return out
+
+
+def profile_case(args):
+    """Small, self-ending cases for ncu captures: every kernel of one ESA step, ``--reps`` times, on
+    inputs larger than L2 but well under a few GB.  Inputs are N(0,1) bf16 drawn on the device."""
+    import paper_2502_14477_b200 as esa
+    H, HG, d, dc = 32, 8, 128, 128
+    g = torch.Generator(device="cuda").manual_seed(0)
+    wq = (torch.randn(dc, H * d, generator=torch.Generator().manual_seed(1)) / (H * d) ** 0.5).numpy()
+    wk = (torch.randn(dc, HG * d, generator=torch.Generator().manual_seed(2)) / (HG * d) ** 0.5).numpy()
+    if args.profile_case == "prefill":
+        l_C, t, B = 512, args.profile_t, 1
+        n = t + l_C
+    else:
+        l_C, t, B = 1, args.profile_t, 8
+        n = t + args.reps + 1
+    ctx = esa.Esa(esa.EsaConfig(H, HG, d, dc, 128, 2048, 4096, 3, l_C, B, n))
+    ctx.set_compressors(wq, None, wk, None)
+    K = torch.randn(B, n, HG, d, device="cuda", dtype=torch.bfloat16, generator=g)
+    V = torch.randn(B, n, HG, d, device="cuda", dtype=torch.bfloat16, generator=g)
+    Q = torch.randn(B, l_C, H, d, device="cuda", dtype=torch.bfloat16, generator=g)
+    Kc = torch.zeros(B, n, dc, dtype=torch.bfloat16, device="cuda")
+    for r0 in range(0, t, 4096):
+        r1 = min(t, r0 + 4096)
+        ctx.compress_keys(K[:, r0:r1].contiguous(), Kc, [r0] * B)
+    idx = torch.zeros(B, 4096, dtype=torch.int32, device="cuda")
+    n_sel = torch.zeros(B, dtype=torch.int32, device="cuda")
+    O = torch.empty_like(Q)
+    torch.cuda.synchronize()
+    ctx.set_profiling(True)
+    for i in range(args.reps):
+        tt = [t + (i if l_C == 1 else 0)] * B
+        ctx.compress_keys(K[:, tt[0]: tt[0] + l_C].contiguous(), Kc, tt)
+        ctx.select(Q, Kc, tt, idx, n_sel)
+        ctx.attend(Q, K, V, tt, idx, n_sel, O)
+    ctx.set_profiling(False)
+    torch.cuda.synchronize()
+    assert ctx.last_device_status() == 0
+    prof = {k: {"launches": n_, "us_per_launch": round(1e3 * ms / n_, 2)} for k, (n_, ms) in ctx.read_profile().items()}
+    print(json.dumps({"profile_case": args.profile_case, "t": t, "reps": args.reps, "launches": ctx.launch_count,
+                      "kernels_isolated": prof}))
 
 
 def run_esa(args, cfg):
@@ -444,16 +600,17 @@ def run_esa(args, cfg):
     for i in range(args.warmup):
         one_step(i)
     sync_all()
+    ctx.read_profile()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     launches0 = ctx.launch_count
-    events = []
+    sampled = []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     e0.record()
     for i in range(args.steps):
-        one_step(args.warmup + i, events)
+        one_step(args.warmup + i, sampled)
     e1.record()
     sync_all()
     ms_total = max_over_ranks(e0.elapsed_time(e1), "cuda" if world > 1 else None)
@@ -463,18 +620,31 @@ def run_esa(args, cfg):
     ms_per_step = ms_total / args.steps
     value = world * cfg.S / (N_LAYERS_STACK * ms_per_step * 1e-3)
 
-    # roofline of the dominant kernel (the attention launches), timed inside the region above
-    att_ms = sum(a.elapsed_time(b) for (_, _, a, b) in events)
+    # rooflines of the kernels, timed inside the region above on the sampled chunks
+    prof = ctx.read_profile()
+    by_kernel = kernel_rooflines(prof, sampled, cfg, peaks)
     n_chunks = (cfg.S + cfg.l_C - 1) // cfg.l_C
-    att_flops = sum(attend_flops(cfg, t, l_C) for (t, l_C, _, _) in events)
-    achieved = att_flops / (att_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (key-list splits merged inside the kernel)", "achieved": achieved, "peak": peaks["tflops_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["tflops_sustained"], "traffic": ATTEND_TC_DRAM_BYTES,
+    att = by_kernel.get("attend_tc_kernel", {"achieved": 0.0, "frac_sustained": 0.0, "frac_burst": 0.0, "launches": 0})
+    att_ms = prof.get("attend_tc_kernel", (0, 0.0))[1]
+    roofline = {"bound": "tensor", "kernel": "attend_tc_kernel (key-list splits merged inside the kernel)",
+                "achieved": att["achieved"], "peak": peaks["tflops_sustained"],
+                "unit": "TFLOP/s", "frac": att["frac_sustained"], "frac_sustained": att["frac_sustained"],
+                "frac_burst": att["frac_burst"], "peak_burst": peaks["tflops_burst"],
+                "traffic": ATTEND_TC_DRAM_BYTES,
                 "traffic_unit": "bytes per attend_tc_kernel launch (ncu, profiles/dram_bytes_per_kernel.txt)",
-                "peak_source": peaks["source"] + " sustained bf16",
-                "share_of_step": att_ms * (args.steps * n_chunks / max(1, len(events))) / ms_total,
-                "launches": len(events),
-                "sampling": "CUDA events around 1 attention launch in %d, position rotating over the steps" % ATTEND_EVENT_EVERY}
+                "peak_source": peaks["source"] + " bf16: sustained (a kernel inside a long step) and burst (the clocks "
+                               "sampled during the run decide which applies: at the maximum SM clock, the burst one)",
+                "share_of_step": att_ms * (args.steps * n_chunks / max(1, len(sampled))) / ms_total,
+                "launches": att["launches"],
+                "sampling": "CUDA events around every kernel of 1 chunk in %d, position rotating over the steps" % PROFILE_EVERY}
+
+    # host time to enqueue a chunk (three library calls + the side-stream bookkeeping), GPU queue empty at the start
+    torch.cuda.synchronize()
+    probe = cfg.with_(S=64 * cfg.l_C)
+    h0 = time.perf_counter()
+    run_prefill_layer(ctx, probe, layers[0], bufs)
+    host_us_per_chunk = 1e6 * (time.perf_counter() - h0) / 64
+    torch.cuda.synchronize()
 
     # end to end: host inputs and outputs
     L0 = layers[0]
@@ -509,15 +679,23 @@ def run_esa(args, cfg):
     decode = None
     if not args.no_decode:
         cfg3 = syn.get_config("c3")
-        us, byts, lps = time_decode(cfg3, args.decode_steps, rank)
+        us, byts, lps, dprof = time_decode(cfg3, args.decode_steps, rank)
         us = max_over_ranks(us, "cuda" if world > 1 else None)
         gbs = byts / (us * 1e-6) / 1e9
         decode = {"workload": "c3: 8 sequences x 131072 cached tokens, 1 query each, k=4096 l_L=2048 l_I=128",
                   "us_per_step": us, "steps": args.decode_steps, "launches_per_step": lps,
+                  "kernels_isolated": dprof,
                   "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": gbs / peaks["hbm_gbs"], "traffic": DECODE_STEP_DRAM_BYTES,
                                "traffic_unit": "bytes per decode step, all kernels (ncu, profiles/dram_bytes_per_kernel.txt)",
                                "algorithmic_bytes_per_step": byts, "peak_source": peaks["source"] + " copy"}}
+
+    # secondary prefill workloads (rank 0's figures are reported; every rank runs them so that the
+    # ranks stay in step)
+    legs = {}
+    if not args.no_legs:
+        for name in ("c2", "c4"):
+            legs["prefill_" + name] = time_prefill_leg(name, 2, peaks)
 
     if rank != 0:
         if world > 1:
@@ -532,9 +710,11 @@ def run_esa(args, cfg):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": workload_config(cfg), "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu, "decode": decode,
+        "roofline": roofline, "roofline_by_kernel": by_kernel, "host_us_per_chunk": host_us_per_chunk,
+        "cpu_baseline": cpu, "decode": decode,
         "per_layer_tokens_per_s": world * cfg.S / (ms_per_step * 1e-3),
     }
+    line.update(legs)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -549,8 +729,18 @@ def main():
     ap.add_argument("--layers", type=int, default=3, help="distinct layers' data kept resident")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the secondary prefill workloads (c2, c4)")
+    ap.add_argument("--profile-case", choices=["prefill", "decode"],
+                    help="run a small self-ending case of every kernel of one step (for ncu captures) and exit")
+    ap.add_argument("--profile-t", type=int, default=65536, help="tokens cached before the profiled chunk / step")
+    ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
     cfg = syn.get_config("c5")
+    if args.profile_case:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py --profile-case needs a CUDA device")
+        profile_case(args)
+        return
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

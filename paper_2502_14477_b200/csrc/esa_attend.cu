@@ -378,29 +378,37 @@ attend_decode_kernel(AttendParams p) {
     const int64_t tok_stride = (int64_t)p.HG * D;
 
     // list positions -> token positions of the rows of iteration `it` that this lane copies
+    // (a position read from the selection is range-checked when it is used, one iteration later, so that
+    // the index load stays in flight meanwhile; sel_mask remembers which rows those are)
     int bad_idx = 0;
+    uint32_t sel_mask = 0;          // rows of the positions looked up last that came from the selection
     auto lookup = [&](int it, int (&pos)[PER_LANE]) {
+        sel_mask = 0;
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) {
             const int j = it * DEC_ROWS + my_row + i * ROWS_PER_PASS;
             int q = -1;
             if (it < it_end && j < n_att) {
                 if (j < i_end) q = j;
-                else if (j < n_glob) q = clamp_selected(__ldg(idx + (j - i_end)), i_end, m_end, bad_idx);
-                else q = m_end + (j - n_glob);
+                else if (j < n_glob) {
+                    q = __ldg(idx + (j - i_end));
+                    sel_mask |= 1u << i;
+                } else q = m_end + (j - n_glob);
             }
             pos[i] = q;
         }
     };
-    auto issue = [&](int stage, const int (&pos)[PER_LANE]) {
+    auto issue = [&](int stage, int (&pos)[PER_LANE], uint32_t mask) {
         uint4* sk = ring + stage * STAGE_CHUNKS;
         uint4* sv = sk + TILE_CHUNKS;
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) {
             const int r = my_row + i * ROWS_PER_PASS;
-            const int64_t off = (int64_t)(pos[i] < 0 ? 0 : pos[i]) * tok_stride;
-            cp_async16(&sk[swz<CH>(r, my_chunk)], Kb + off, pos[i] < 0 ? 0 : 16);
-            cp_async16(&sv[swz<CH>(r, my_chunk)], Vb + off, pos[i] < 0 ? 0 : 16);
+            int q = pos[i];
+            if ((mask >> i) & 1u) q = clamp_selected(q, i_end, m_end, bad_idx);
+            const int64_t off = (int64_t)(q < 0 ? 0 : q) * tok_stride;
+            cp_async16(&sk[swz<CH>(r, my_chunk)], Kb + off, q < 0 ? 0 : 16);
+            cp_async16(&sv[swz<CH>(r, my_chunk)], Vb + off, q < 0 ? 0 : 16);
         }
     };
 
@@ -431,14 +439,14 @@ attend_decode_kernel(AttendParams p) {
 #pragma unroll
     for (int s = 0; s < DEC_STAGES - 1; ++s) {
         lookup(it0 + s * DEC_WARPS, pos_next);
-        issue(s, pos_next);
+        issue(s, pos_next, sel_mask);
         cp_async_commit();
     }
     lookup(it0 + (DEC_STAGES - 1) * DEC_WARPS, pos_next);
 
     int n = 0;
     for (int it = it0; it < it_end; it += DEC_WARPS, ++n) {
-        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next);
+        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next, sel_mask);
         cp_async_commit();
         lookup(it + DEC_STAGES * DEC_WARPS, pos_next);
         cp_async_wait<DEC_STAGES - 1>();

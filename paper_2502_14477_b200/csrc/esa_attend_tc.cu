@@ -565,16 +565,24 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             const uint32_t ph = ((j / TC_STAGES) & 1) ^ 1;
             const int key0 = (tile_begin + j) * TC_BN;
             int pos[TC_BN / RSTEP];
+            uint32_t from_idx = 0;                      // rows whose position was read from the selection
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int jj = key0 + rsub + it * RSTEP;
                 int q = -1;
                 if (jj < i_end) q = jj;
-                else if (jj < n_glob) q = clamp_selected(__ldg(idx + (jj - i_end)), i_end, m_end, bad_idx);
-                else if (jj < n_att) q = m_end + (jj - n_glob);
+                else if (jj < n_glob) {
+                    q = __ldg(idx + (jj - i_end));
+                    from_idx |= 1u << it;
+                } else if (jj < n_att) q = m_end + (jj - n_glob);
                 pos[it] = q;
             }
             mbar_wait(bar(BAR_K_EMPTY + s), ph, wc);
+            // (the range check of the selected positions comes after the wait: the index loads above stay in
+            // flight across it instead of being consumed at once)
+#pragma unroll
+            for (int it = 0; it < TC_BN / RSTEP; ++it)
+                if ((from_idx >> it) & 1u) pos[it] = clamp_selected(pos[it], i_end, m_end, bad_idx);
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int r = rsub + it * RSTEP;

@@ -11,7 +11,7 @@
 // The selection kernel starts from the pooled keys and the histogram of their top 11 bits
 // (both left by the scoring kernels, or by pool_hist_kernel below for the scoring paths that
 // do not pool).  It runs in two phases inside one launch, and no CTA ever waits for another:
-//   1. every CTA owns a slice of 4096 consecutive tokens.  From the histogram it finds the bin
+//   1. every CTA owns a slice of 8192 consecutive tokens.  From the histogram it finds the bin
 //      b0 that holds the k-th largest key, and copies the keys that can still matter -- those
 //      not below the lower edge of b0 -- with their positions, in index order, to its slice of
 //      a candidate list; then it draws an arrival ticket.
@@ -28,12 +28,12 @@
 
 namespace esa {
 
-constexpr int SEL_THREADS = 512;
-constexpr int SEL_SLICE = 4096;       // tokens per CTA in phase 1
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_SLICE = 8192;       // tokens per CTA in phase 1
 constexpr int SEL_PER = SEL_SLICE / SEL_THREADS;
 constexpr int SEL_ROWS = SEL_SLICE / 32;
 constexpr int SEL_BINS = 2048;
-constexpr int SEL_STAGE_CAP = 16384;  // candidates the last CTA can stage in shared memory
+constexpr int SEL_STAGE_CAP = 12288;  // candidates the last CTA can stage in shared memory (keys and positions)
 constexpr int SEL_MAX_SLICES_SMEM = 1024;
 
 struct SelectParams {
@@ -149,7 +149,7 @@ select_topk_kernel(SelectParams p) {
     const int slice = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    extern __shared__ uint32_t sel_dyn[];          // last CTA: slice offsets, then the staged candidate keys
+    extern __shared__ uint32_t sel_dyn[];          // last CTA: slice offsets, then the staged candidate keys and positions
     __shared__ uint32_t hist[SEL_BINS];
     __shared__ int row_cnt[SEL_THREADS];           // phase 1: candidates per 32-token row; phase 2: slice offsets (first part)
     __shared__ int warp_tot[33];
@@ -231,36 +231,70 @@ select_topk_kernel(SelectParams p) {
     // SEL_MAX_SLICES_SMEM offsets; longer sequences re-read the counts)
     int* soff = reinterpret_cast<int*>(sel_dyn);   // [n_slices + 1] when it fits, ahead of the staged candidates
     const bool offs_in_smem = n_slices + 1 <= SEL_MAX_SLICES_SMEM;
-    int total = 0;
-    for (int s0 = 0; s0 < n_slices; s0 += SEL_THREADS) {
-        const int s = s0 + tid;
-        const int c = s < n_slices ? __ldcg(p.slice_cnt + (int64_t)b * p.slice_stride + s) : 0;
-        row_cnt[tid] = c;
-        __syncthreads();
-        const int t = block_exclusive_scan(row_cnt, SEL_THREADS, warp_tot);
-        if (offs_in_smem && s < n_slices) soff[s] = total + row_cnt[tid];
-        total += t;
-        __syncthreads();
+    if (warp == 0) {
+        // one warp scans the slice counts, 32 per round (a sequence has a few dozen slices)
+        int run = 0;
+        for (int s0 = 0; s0 < n_slices; s0 += 32) {
+            const int s = s0 + lane;
+            const int c = s < n_slices ? __ldcg(p.slice_cnt + (int64_t)b * p.slice_stride + s) : 0;
+            int incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int x = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += x;
+            }
+            if (offs_in_smem && s < n_slices) soff[s] = run + incl - c;
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            if (offs_in_smem) soff[n_slices] = run;
+            warp_tot[32] = run;
+        }
     }
-    if (offs_in_smem && tid == 0) soff[n_slices] = total;
     __syncthreads();
+    const int total = warp_tot[32];
     const int C = total;                           // >= k candidates in all
     uint32_t* skeys = sel_dyn + SEL_MAX_SLICES_SMEM;
+    int32_t* sidx = reinterpret_cast<int32_t*>(skeys + SEL_STAGE_CAP);
     const bool staged = offs_in_smem && C <= SEL_STAGE_CAP;
     const uint32_t* dk;
-    // where candidate i of the dense order lives in the per-slice lists: the slice s with soff[s] <= i < soff[s + 1]
-    auto src_of = [&](int i) {
-        int lo = 0, hi = n_slices;                     // invariant: soff[lo] <= i < soff[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (soff[mid] <= i) lo = mid; else hi = mid;
-        }
-        return lo * SEL_SLICE + (i - soff[lo]);
-    };
+    const int32_t* di;
     if (staged) {
-        // dense copy of the keys in shared memory (the positions are fetched for the selected ones only)
-        for (int i = tid; i < C; i += SEL_THREADS) skeys[i] = __ldcg(ck + src_of(i));
+        // dense copy in shared memory: candidate i of the dense order lives in the slice s with
+        // soff[s] <= i < soff[s + 1].  Eight candidates per thread and round, their sixteen loads in flight together.
+        auto src_of = [&](int i) {
+            int lo = 0, hi = n_slices;                     // invariant: soff[lo] <= i < soff[hi]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (soff[mid] <= i) lo = mid; else hi = mid;
+            }
+            return lo * SEL_SLICE + (i - soff[lo]);
+        };
+        for (int i0 = tid; i0 < C; i0 += 8 * SEL_THREADS) {
+            int src[8];
+            uint32_t kk[8];
+            int32_t ii[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * SEL_THREADS;
+                src[u] = i < C ? src_of(i) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                kk[u] = __ldcg(ck + src[u]);
+                ii[u] = __ldcg(ci + src[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * SEL_THREADS;
+                if (i < C) {
+                    skeys[i] = kk[u];
+                    sidx[i] = ii[u];
+                }
+            }
+        }
         dk = skeys;
+        di = sidx;
     } else {
         // too many candidates (long runs of equal scores): close the gaps in place, slice by slice
         // (a slice's list moves to a lower or equal address; it is read into registers first)
@@ -288,6 +322,7 @@ select_topk_kernel(SelectParams p) {
             __syncthreads();
         }
         dk = ck;
+        di = ci;
     }
     __syncthreads();
 
@@ -371,7 +406,7 @@ select_topk_kernel(SelectParams p) {
         const uint32_t my_eq = eq_before + __popc(be & lt_mask);
         if (gt || (eq && my_eq < take_eq)) {
             const uint32_t pos = my_gt + min(my_eq, take_eq);
-            if (pos < (uint32_t)k) out[pos] = staged ? __ldcg(ci + src_of(i)) : ci[i];
+            if (pos < (uint32_t)k) out[pos] = di[i];
         }
         gt_before += __popc(bg);
         eq_before += __popc(be);
@@ -462,7 +497,7 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.slice_stride = ctx->sel_slice_stride; p.top_k = ctx->cfg.top_k;
     p.mapped = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
-    constexpr size_t smem = (size_t)(SEL_MAX_SLICES_SMEM + SEL_STAGE_CAP) * 4;
+    constexpr size_t smem = (size_t)(SEL_MAX_SLICES_SMEM + 2 * SEL_STAGE_CAP) * 4;
     e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     ProfScope prof(ctx, KC_SELECT_TOPK, st);
