@@ -146,6 +146,26 @@ esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
                             const void* K_cache, const void* V_cache, const int64_t* n_prev,
                             const int32_t* idx, const int32_t* n_sel, void* O, void* stream);
 
+/* Section 3.2 (position encoding) / Algorithm 1 with two encodings of the same tokens.  The
+ * paper attends I and M_k at one fixed distance (the queries of C encoded at a fixed position
+ * w, those keys at position 0) and L and C at their true relative positions, and normalises
+ * over both parts together.  The rotation itself stays with the caller; this call takes the two
+ * encodings as separate tensors:
+ *   Q_cur       device [B, l_C, H, d]             queries used against L and C
+ *   Q_far       device [B, l_C, H, d] or NULL     queries used against I and M_k   (NULL: Q_cur)
+ *   K_cache     device [B, max_tokens, H_G, d]    keys read for L and C
+ *   K_far_cache device [B, max_tokens, H_G, d] or NULL   keys read for I and M_k  (NULL: K_cache)
+ * One softmax spans the logits of both parts (Algorithm 1's merge of its two partial results by
+ * their normalisers); values come from V_cache for every key.  Everything else is as for
+ * esa_attend, which is this call with both optional tensors NULL. */
+esa_status esa_attend_two_position(esa_ctx* ctx, int32_t B, const void* Q_cur, const void* Q_far, int32_t l_C,
+                                   const void* K_cache, const void* K_far_cache, const void* V_cache,
+                                   const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel, void* O);
+esa_status esa_attend_two_position_async(esa_ctx* ctx, int32_t B, const void* Q_cur, const void* Q_far, int32_t l_C,
+                                         const void* K_cache, const void* K_far_cache, const void* V_cache,
+                                         const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel, void* O,
+                                         void* stream);
+
 /* (No counterpart in the paper: an integration convenience.)
  * esa_attend for small chunks -- l_C * (H / H_G) <= 64 rows, the decode case -- that needs
  * neither a context nor any allocation.  It is for callers that may not allocate device

@@ -25,7 +25,8 @@ compressor weights are rounded once to bf16; q' and k' are accumulated exactly
 in fp32; attention runs in float64 on the bf16 inputs.
 
 Pins (tests/test_oracle_pins.py): attention == textbook causal attention when
-k >= l_M; Algorithm 1's two-part LSE merge == one softmax over the union;
+k >= l_M; part-by-part attention merged by log-normalisers (Algorithm 1) == one
+softmax over the union, also with distinct far/near queries and keys (Section 3.2);
 scores/aggregate/top-k == brute-force loops on tiny inputs; proximity_pool ==
 a library 1-D max pool; compress == plain matrix product and the GQA folding
 identity; the flop/cache closed forms reproduce the paper's 1.56 % and 6.25 %.
@@ -155,19 +156,30 @@ def attend_positions(t: int, l_C: int, sel_abs: np.ndarray, p: EsaParams) -> np.
 
 
 def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t: int,
-           p: EsaParams, return_lse: bool = False, heads=None):
+           p: EsaParams, return_lse: bool = False, heads=None, Q_global=None, K_global=None):
     """Eq. 1.  Q_C [l_C,H,d]; K,V [>=t+l_C,H_G,d] with C at [t,t+l_C);
     sel_abs absolute positions of the selected middle tokens.  Query head h
     uses key/value head h // (H/H_G).  Query c sees every I, M_k and L key and
     the C keys at chunk offsets <= c (Algorithm 1: non-causal on [I,M_k],
     causal with bottom-right alignment on [L,C]).  Returns float64 [l_C,H,d];
-    with ``heads`` given only those query heads are computed (the rest are NaN)."""
+    with ``heads`` given only those query heads are computed (the rest are NaN).
+
+    Section 3.2 (two positions): the logits against I and M_k may use a second
+    encoding of the same tokens -- queries ``Q_global`` (all at one fixed
+    position) and keys ``K_global`` (all at position 0) -- while the logits
+    against L and C use Q_C and K (relative positions).  The softmax still spans
+    the union of both sets of logits, which is what Algorithm 1's weighting of
+    its two partial results by their normalisers amounts to.  None = the same
+    tensors for both parts."""
     Q_C = np.asarray(Q_C, np.float64)
+    Qg = Q_C if Q_global is None else np.asarray(Q_global, np.float64)
+    Kg = K if K_global is None else K_global
     l_C, H, d = Q_C.shape
     H_G = K.shape[1]
     g = H // H_G
     scale = p.scale if p.scale > 0 else 1.0 / np.sqrt(d)
     pos = attend_positions(t, l_C, sel_abs, p)
+    i_far = partition(t, p.l_I, p.l_L)[0] + len(sel_abs)   # |I| + |M_k|
     n_prev = pos.shape[0] - l_C                      # keys before C in the list
     # visible[c, j]: every key before C; C key u visible iff u <= c
     visible = np.ones((l_C, pos.shape[0]), dtype=bool)
@@ -175,9 +187,11 @@ def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t
     O = np.full((l_C, H, d), np.nan, np.float64)
     LSE = np.full((l_C, H), np.nan, np.float64)
     for h in (range(H) if heads is None else heads):
-        Kh = np.asarray(K[pos, h // g, :], np.float64)
         Vh = np.asarray(V[pos, h // g, :], np.float64)
-        logits = scale * (Q_C[:, h, :] @ Kh.T)
+        n_far = i_far                                        # list entries of I and M_k come first
+        logits = np.concatenate(
+            [scale * (Qg[:, h, :] @ np.asarray(Kg[pos[:n_far], h // g, :], np.float64).T),
+             scale * (Q_C[:, h, :] @ np.asarray(K[pos[n_far:], h // g, :], np.float64).T)], axis=1)
         logits = np.where(visible, logits, -np.inf)
         mx = logits.max(axis=1, keepdims=True)
         w = np.exp(logits - mx)
@@ -187,44 +201,67 @@ def attend(Q_C: np.ndarray, K: np.ndarray, V: np.ndarray, sel_abs: np.ndarray, t
     return (O, LSE) if return_lse else O
 
 
-def _softmax_part(Qh, Kh, Vh, scale, mask):
+def softmax_part(Qh, Kh, Vh, scale, mask=None):
+    """Attention of the rows of Qh over one set of keys on its own: (normalised output, log of
+    the normaliser).  A row that sees no key gives (0, -inf)."""
     logits = scale * (Qh @ Kh.T)
     if mask is not None:
         logits = np.where(mask, logits, -np.inf)
+    if logits.shape[1] == 0:
+        return np.zeros((Qh.shape[0], Vh.shape[1])), np.full(Qh.shape[0], -np.inf)
     mx = logits.max(axis=1, keepdims=True)
+    mx = np.where(np.isfinite(mx), mx, 0.0)
     w = np.exp(logits - mx)
     den = w.sum(axis=1, keepdims=True)
-    return (w / den) @ Vh, (mx + np.log(den))[:, 0]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        out = np.where(den > 0, (w @ Vh) / den, 0.0)
+        lse = np.where(den[:, 0] > 0, mx[:, 0] + np.log(den[:, 0]), -np.inf)
+    return out, lse
 
 
-def attend_alg1(Q_C, K, V, sel_abs, t, p: EsaParams):
-    """Algorithm 1 with identical local and global queries: a causal call on
-    [L,C], a non-causal call on [I,M_k], merged with weights
-    softmax([lse_local, lse_global]) (the exponentials taken after subtracting
-    the larger lse)."""
+def merge_softmax_parts(parts):
+    """Attention over a union of disjoint key sets from the per-set results: each part is
+    (normalised output [n, d], log-normaliser [n]); the union's output is the parts' outputs
+    weighted by softmax over the parts of their log-normalisers (taken after subtracting the
+    largest one).  With two parts this is the weighting step of the paper's Algorithm 1."""
+    lse = np.stack([q for _, q in parts], axis=0)               # [parts, n]
+    top = lse.max(axis=0, keepdims=True)
+    top = np.where(np.isfinite(top), top, 0.0)
+    w = np.exp(lse - top)
+    w = w / w.sum(axis=0, keepdims=True)
+    return sum(wi[:, None] * o for wi, (o, _) in zip(w, parts))
+
+
+def attend_by_parts(Q_C, K, V, sel_abs, t, p: EsaParams, Q_global=None, K_global=None, cuts=None):
+    """The same attention as ``attend`` computed part by part: the key list is cut into pieces
+    (by default the two of Algorithm 1: [I, M_k] seen by the far-position queries without a causal
+    mask, [L, C] seen by the near-position queries causally), each piece is attended on its own,
+    and the pieces are merged by ``merge_softmax_parts``.  ``cuts`` gives other cut points inside
+    the key list (any piece lying in the first |I|+|M_k| entries uses the far-position tensors)."""
     Q_C = np.asarray(Q_C, np.float64)
+    Qg = Q_C if Q_global is None else np.asarray(Q_global, np.float64)
+    Kg = K if K_global is None else K_global
     l_C, H, d = Q_C.shape
     g = H // K.shape[1]
     scale = p.scale if p.scale > 0 else 1.0 / np.sqrt(d)
-    i_end, m_end = partition(t, p.l_I, p.l_L)
-    gpos = np.concatenate([np.arange(0, i_end), np.asarray(sel_abs, np.int64)]).astype(np.int64)
-    lpos = np.arange(m_end, t + l_C)
-    n_L = t - m_end
-    lmask = np.ones((l_C, lpos.shape[0]), dtype=bool)
-    lmask[:, n_L:] = np.tril(np.ones((l_C, l_C), dtype=bool))
+    pos = attend_positions(t, l_C, sel_abs, p)
+    n_far = partition(t, p.l_I, p.l_L)[0] + len(sel_abs)
+    n_prev = pos.shape[0] - l_C
+    visible = np.ones((l_C, pos.shape[0]), dtype=bool)
+    visible[:, n_prev:] = np.tril(np.ones((l_C, l_C), dtype=bool))
+    edges = sorted(set([0, n_far, pos.shape[0]] + list(cuts or [])))
     O = np.empty((l_C, H, d), np.float64)
     for h in range(H):
-        Qh = Q_C[:, h, :]
-        l_attn, l_lse = _softmax_part(Qh, np.asarray(K[lpos, h // g], np.float64),
-                                      np.asarray(V[lpos, h // g], np.float64), scale, lmask)
-        if gpos.shape[0] == 0:
-            O[:, h, :] = l_attn
-            continue
-        g_attn, g_lse = _softmax_part(Qh, np.asarray(K[gpos, h // g], np.float64),
-                                      np.asarray(V[gpos, h // g], np.float64), scale, None)
-        top = np.maximum(l_lse, g_lse)
-        se_l, se_g = np.exp(l_lse - top), np.exp(g_lse - top)
-        O[:, h, :] = (l_attn * se_l[:, None] + g_attn * se_g[:, None]) / (se_l + se_g)[:, None]
+        parts = []
+        for a, b in zip(edges[:-1], edges[1:]):
+            if a == b:
+                continue
+            far = b <= n_far
+            Qh = (Qg if far else Q_C)[:, h, :]
+            Kh = np.asarray((Kg if far else K)[pos[a:b], h // g], np.float64)
+            Vh = np.asarray(V[pos[a:b], h // g], np.float64)
+            parts.append(softmax_part(Qh, Kh, Vh, scale, visible[:, a:b]))
+        O[:, h, :] = merge_softmax_parts(parts)
     return O
 
 

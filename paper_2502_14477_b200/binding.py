@@ -82,6 +82,11 @@ _PROTOS = {
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_attend_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_attend_two_position": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_attend_two_position_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                C.c_void_p]),
     "esa_attend_noalloc": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_read_pooled_scores": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
@@ -278,6 +283,32 @@ class Esa:
                                            _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_attend")
+
+    def attend_two_position(self, Q_cur, Q_far, K_cache, K_far_cache, V_cache, n_prev, idx, n_sel, O, stream=None,
+                            sync=False):
+        """``esa_attend_two_position``: Q_far / K_far_cache (either may be None) are read for I and M_k."""
+        c = self.cfg
+        B, l_C = Q_cur.shape[0], Q_cur.shape[1]
+        _check(Q_cur, "Q_cur", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        if Q_far is not None:
+            _check(Q_far, "Q_far", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        _check(K_cache, "K_cache", torch.bfloat16, (B, c.max_tokens, c.n_kv_heads, c.head_dim))
+        if K_far_cache is not None:
+            _check(K_far_cache, "K_far_cache", torch.bfloat16, (B, c.max_tokens, c.n_kv_heads, c.head_dim))
+        _check(V_cache, "V_cache", torch.bfloat16, (B, c.max_tokens, c.n_kv_heads, c.head_dim))
+        _check(idx, "idx", torch.int32, (B, c.top_k))
+        _check(n_sel, "n_sel", torch.int32, (B,))
+        _check(O, "O", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        npv = self._nprev(n_prev, B)
+        if sync:
+            st = self.lib.esa_attend_two_position(self._h, B, _ptr(Q_cur), _ptr(Q_far), l_C, _ptr(K_cache),
+                                                  _ptr(K_far_cache), _ptr(V_cache), npv, _ptr(idx), _ptr(n_sel), _ptr(O))
+        else:
+            st = self.lib.esa_attend_two_position_async(self._h, B, _ptr(Q_cur), _ptr(Q_far), l_C, _ptr(K_cache),
+                                                        _ptr(K_far_cache), _ptr(V_cache), npv, _ptr(idx), _ptr(n_sel),
+                                                        _ptr(O), _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_attend_two_position")
 
     def read_pooled_scores(self, b: int, n: int, stream=None) -> np.ndarray:
         out = np.empty(n, dtype=np.float32)

@@ -361,9 +361,10 @@ esa_status esa_select(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, c
 }
 
 // -------------------------------------------------------------------- attend
-esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
-                            const void* V_cache, const int64_t* n_prev, const int32_t* idx,
-                            const int32_t* n_sel, void* O, void* stream) {
+esa_status esa_attend_two_position_async(esa_ctx* ctx, int32_t B, const void* Q_cur, const void* Q_far, int32_t l_C,
+                                         const void* K_cache, const void* K_far_cache, const void* V_cache,
+                                         const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel, void* O,
+                                         void* stream) {
     esa_status s = check_common(ctx, B);
     if (s != ESA_OK) return s;
     if (!Q_cur || !K_cache || !V_cache || !n_prev || !idx || !n_sel || !O || l_C <= 0) return ESA_ERR_INVALID_ARG;
@@ -371,9 +372,26 @@ esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     SeqMeta meta;
     s = build_meta(ctx, B, n_prev, l_C, &meta, nullptr);
     if (s != ESA_OK) return s;
-    return from_cuda(launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)K_cache,
+    return from_cuda(launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)Q_far,
+                                   (const __nv_bfloat16*)K_cache, (const __nv_bfloat16*)K_far_cache,
                                    (const __nv_bfloat16*)V_cache, meta, idx, n_sel, (__nv_bfloat16*)O,
                                    (cudaStream_t)stream));
+}
+
+esa_status esa_attend_two_position(esa_ctx* ctx, int32_t B, const void* Q_cur, const void* Q_far, int32_t l_C,
+                                   const void* K_cache, const void* K_far_cache, const void* V_cache,
+                                   const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel, void* O) {
+    esa_status s = esa_attend_two_position_async(ctx, B, Q_cur, Q_far, l_C, K_cache, K_far_cache, V_cache, n_prev, idx,
+                                                 n_sel, O, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
+esa_status esa_attend_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                            const void* V_cache, const int64_t* n_prev, const int32_t* idx,
+                            const int32_t* n_sel, void* O, void* stream) {
+    return esa_attend_two_position_async(ctx, B, Q_cur, nullptr, l_C, K_cache, nullptr, V_cache, n_prev, idx, n_sel, O,
+                                         stream);
 }
 
 esa_status esa_attend(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,

@@ -29,6 +29,8 @@ namespace esa {
 struct AttendParams {
     const __nv_bfloat16* Q;   // [B, l_C, H, D]
     const __nv_bfloat16* K;   // [B, max_tokens, HG, D]
+    const __nv_bfloat16* Qg;  // two-position attention (Section 3.2): queries / keys used against I and M_k
+    const __nv_bfloat16* Kg;  //   (equal to Q / K otherwise)
     const __nv_bfloat16* V;
     __nv_bfloat16* O;         // [B, l_C, H, D]
     const int32_t* idx;       // [B, top_k]
@@ -46,7 +48,9 @@ struct AttendParams {
 // layout of the split-KV partial buffer, per (b, kvh, split): R rows x (D + 2) floats
 // (unnormalised O row, running max m in the exp2 domain, running sum l)
 
-template <int D, int NW, int BN>
+// TWO: the list entries of I and M_k (the first n_glob) take their logits from Qg and Kg, the entries
+// of L and C from Q and K; both score tiles are formed and each key column keeps the one that applies.
+template <int D, int NW, int BN, bool TWO>
 __global__ void __launch_bounds__(NW * 32)
 attend_kernel(AttendParams p) {
     constexpr int CH = D / 8;
@@ -56,6 +60,7 @@ attend_kernel(AttendParams p) {
     uint4* sQ = smem;                         // [BM][CH]
     uint4* sK = sQ + BM * CH;                 // 2 x [BN][CH]
     uint4* sV = sK + 2 * BN * CH;             // 2 x [BN][CH]
+    uint4* sQg = sV + 2 * BN * CH;            // [BM][CH] (TWO)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row0 = blockIdx.x * BM;
@@ -81,6 +86,7 @@ attend_kernel(AttendParams p) {
     const int tile_end = min(n_tiles, tile_begin + per);
 
     const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D;
+    const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D;
     const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D;
     const int32_t* idx = p.idx + (int64_t)b * p.top_k;
     const int64_t tok_stride = (int64_t)p.HG * D;
@@ -100,7 +106,7 @@ attend_kernel(AttendParams p) {
                 else pos = m_end + (j - n_glob);
             }
             const int64_t off = (int64_t)pos * tok_stride + c * 8;
-            cp_async16(&dk[swz<CH>(r, c)], Kb + off, ok ? 16 : 0);
+            cp_async16(&dk[swz<CH>(r, c)], ((TWO && j < n_glob) ? Kgb : Kb) + off, ok ? 16 : 0);
             cp_async16(&dv[swz<CH>(r, c)], Vb + off, ok ? 16 : 0);
         }
     };
@@ -111,8 +117,9 @@ attend_kernel(AttendParams p) {
         int row = row0 + r;
         bool ok = row < R;
         int cq = ok ? row / G : 0, g = ok ? row % G : 0;
-        const __nv_bfloat16* src = p.Q + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + c * 8;
-        cp_async16(&sQ[swz<CH>(r, c)], src, ok ? 16 : 0);
+        const int64_t qoff = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + c * 8;
+        cp_async16(&sQ[swz<CH>(r, c)], p.Q + qoff, ok ? 16 : 0);
+        if (TWO) cp_async16(&sQg[swz<CH>(r, c)], p.Qg + qoff, ok ? 16 : 0);
     }
     if (tile_begin < tile_end) load_kv(0, tile_begin);
     cp_async_commit();
@@ -132,6 +139,7 @@ attend_kernel(AttendParams p) {
     const int warp_min_lim = c_first + min((row0 + warp * 16) / G, p.l_C - 1) + 1;
 
     uint32_t qf[D / 16][4];
+    uint32_t qfg[TWO ? D / 16 : 1][4];
     bool q_loaded = false;
 
     for (int tile = tile_begin; tile < tile_end; ++tile) {
@@ -147,6 +155,10 @@ attend_kernel(AttendParams p) {
         if (!q_loaded) {
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) load_a_frag<CH>(qf[ks], sQ, warp * 16, ks * 2, lane);
+            if (TWO) {
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) load_a_frag<CH>(qfg[ks], sQg, warp * 16, ks * 2, lane);
+            }
             q_loaded = true;
         }
         const uint4* tk = sK + st * BN * CH;
@@ -168,9 +180,35 @@ attend_kernel(AttendParams p) {
                 mma_bf16_16816(s[2 * nb + 1], qf[ks], kb[2], kb[3]);
             }
         }
+        const int j0 = tile * BN;
+        if (TWO && j0 < n_glob) {
+            // some key columns of this tile belong to I or M_k: their logits come from Qg (the tile holds Kg rows there)
+            float sg[BN / 8][4];
+#pragma unroll
+            for (int i = 0; i < BN / 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) sg[i][j] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+                for (int nb = 0; nb < BN / 16; ++nb) {
+                    uint32_t kb[4];
+                    load_b_frag_nk<CH>(kb, tk, nb * 16, ks * 2, lane);
+                    mma_bf16_16816(sg[2 * nb], qfg[ks], kb[0], kb[1]);
+                    mma_bf16_16816(sg[2 * nb + 1], qfg[ks], kb[2], kb[3]);
+                }
+            }
+#pragma unroll
+            for (int nb = 0; nb < BN / 8; ++nb)
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (j0 + nb * 8 + (lane & 3) * 2 + e < n_glob) {
+                        s[nb][e] = sg[nb][e];
+                        s[nb][2 + e] = sg[nb][2 + e];
+                    }
+        }
 
         // scale, mask (causal inside C and the ragged tail), online softmax
-        const int j0 = tile * BN;
         const bool need_mask = j0 + BN > warp_min_lim;
         float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
@@ -344,7 +382,7 @@ constexpr int DEC_WARPS = 4;
 constexpr int DEC_STAGES = 3;
 constexpr int DEC_ROWS = 16;       // rows (keys) per stage
 
-template <int D, int G>
+template <int D, int G, bool TWO>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 attend_decode_kernel(AttendParams p) {
     constexpr int CH = D / 8;                        // 16-byte chunks per row
@@ -373,6 +411,7 @@ attend_decode_kernel(AttendParams p) {
 
     const int my_chunk = lane % CH, my_row = lane / CH;     // copies of this lane: rows my_row + i * ROWS_PER_PASS
     const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
+    const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
     const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
     const int32_t* idx = p.idx + (int64_t)b * p.top_k;
     const int64_t tok_stride = (int64_t)p.HG * D;
@@ -382,11 +421,14 @@ attend_decode_kernel(AttendParams p) {
     // the index load stays in flight meanwhile; sel_mask remembers which rows those are)
     int bad_idx = 0;
     uint32_t sel_mask = 0;          // rows of the positions looked up last that came from the selection
+    uint32_t far_mask = 0;          // rows of the positions looked up last that belong to I or M_k (TWO: their keys come from Kg)
     auto lookup = [&](int it, int (&pos)[PER_LANE]) {
         sel_mask = 0;
+        far_mask = 0;
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) {
             const int j = it * DEC_ROWS + my_row + i * ROWS_PER_PASS;
+            if (TWO && j < n_glob) far_mask |= 1u << i;
             int q = -1;
             if (it < it_end && j < n_att) {
                 if (j < i_end) q = j;
@@ -398,7 +440,7 @@ attend_decode_kernel(AttendParams p) {
             pos[i] = q;
         }
     };
-    auto issue = [&](int stage, int (&pos)[PER_LANE], uint32_t mask) {
+    auto issue = [&](int stage, int (&pos)[PER_LANE], uint32_t mask, uint32_t fmask) {
         uint4* sk = ring + stage * STAGE_CHUNKS;
         uint4* sv = sk + TILE_CHUNKS;
 #pragma unroll
@@ -407,21 +449,27 @@ attend_decode_kernel(AttendParams p) {
             int q = pos[i];
             if ((mask >> i) & 1u) q = clamp_selected(q, i_end, m_end, bad_idx);
             const int64_t off = (int64_t)(q < 0 ? 0 : q) * tok_stride;
-            cp_async16(&sk[swz<CH>(r, my_chunk)], Kb + off, q < 0 ? 0 : 16);
+            cp_async16(&sk[swz<CH>(r, my_chunk)], ((TWO && ((fmask >> i) & 1u)) ? Kgb : Kb) + off, q < 0 ? 0 : 16);
             cp_async16(&sv[swz<CH>(r, my_chunk)], Vb + off, q < 0 ? 0 : 16);
         }
     };
 
     // B fragments of Q^T for every 16-wide slice of D: element (k = d, n = head); heads >= G are zero
     uint32_t qb[D / 16][2];
+    uint32_t qbg[TWO ? D / 16 : 1][2];      // the same for the queries used against I and M_k
     {
         const int head = lane >> 2;
-        const __nv_bfloat16* qrow = p.Q + ((int64_t)b * p.H + kvh * G + (head < G ? head : 0)) * D;
+        const int64_t qoff = ((int64_t)b * p.H + kvh * G + (head < G ? head : 0)) * D;
+        const __nv_bfloat16* qrow = p.Q + qoff;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
             const int d0 = ks * 16 + 2 * (lane & 3);
             qb[ks][0] = head < G ? *reinterpret_cast<const uint32_t*>(qrow + d0) : 0u;
             qb[ks][1] = head < G ? *reinterpret_cast<const uint32_t*>(qrow + d0 + 8) : 0u;
+            if (TWO) {
+                qbg[ks][0] = head < G ? *reinterpret_cast<const uint32_t*>(p.Qg + qoff + d0) : 0u;
+                qbg[ks][1] = head < G ? *reinterpret_cast<const uint32_t*>(p.Qg + qoff + d0 + 8) : 0u;
+            }
         }
     }
     // this thread's two heads (columns 2 (lane & 3), +1): running maximum and its share of the sum;
@@ -439,14 +487,14 @@ attend_decode_kernel(AttendParams p) {
 #pragma unroll
     for (int s = 0; s < DEC_STAGES - 1; ++s) {
         lookup(it0 + s * DEC_WARPS, pos_next);
-        issue(s, pos_next, sel_mask);
+        issue(s, pos_next, sel_mask, far_mask);
         cp_async_commit();
     }
     lookup(it0 + (DEC_STAGES - 1) * DEC_WARPS, pos_next);
 
     int n = 0;
     for (int it = it0; it < it_end; it += DEC_WARPS, ++n) {
-        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next, sel_mask);
+        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next, sel_mask, far_mask);
         cp_async_commit();
         lookup(it + DEC_STAGES * DEC_WARPS, pos_next);
         cp_async_wait<DEC_STAGES - 1>();
@@ -464,6 +512,18 @@ attend_decode_kernel(AttendParams p) {
         }
         // rows lane / 4 and + 8 of the tile; list positions past the end are masked
         const int key_lo = it * DEC_ROWS + (lane >> 2);
+        if (TWO && it * DEC_ROWS < n_glob) {
+            // rows of I and M_k: logits against the other query encoding (uniform branch over the warp)
+            float sg[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                uint32_t a[4];
+                load_a_frag<CH>(a, tk, 0, ks * 2, lane);
+                mma_bf16_16816(sg, a, qbg[ks][0], qbg[ks][1]);
+            }
+            if (key_lo < n_glob) { sc[0] = sg[0]; sc[1] = sg[1]; }
+            if (key_lo + 8 < n_glob) { sc[2] = sg[2]; sc[3] = sg[3]; }
+        }
         const bool ok_lo = key_lo < n_att, ok_hi = key_lo + 8 < n_att;
         sc[0] = ok_lo ? sc[0] * p.scale_log2 : -INFINITY;
         sc[1] = ok_lo ? sc[1] * p.scale_log2 : -INFINITY;
@@ -586,14 +646,14 @@ attend_decode_kernel(AttendParams p) {
     }
 }
 
-template <int D, int G>
+template <int D, int G, bool TWO>
 static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
     constexpr int smem = DEC_WARPS * DEC_STAGES * 2 * DEC_ROWS * D * 2;
     static_assert(smem >= (2 * DEC_WARPS * 8 + DEC_WARPS * 8 * D) * 4, "the warp merge reuses the rings");
-    cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel<D, G, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int per_sm = 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_decode_kernel<D, G>, DEC_WARPS * 32, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_decode_kernel<D, G, TWO>, DEC_WARPS * 32, smem);
     if (e != cudaSuccess) return e;
     const int iters = (n_att_max + DEC_ROWS - 1) / DEC_ROWS;
     // one wave of CTAs, each warp with at least a few iterations
@@ -606,36 +666,36 @@ static cudaError_t launch_decode_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     if ((size_t)B * p.HG > ctx->att_count_elems) return cudaErrorInvalidConfiguration;
     p.unit_count = ctx->att_count;
     ProfScope prof(ctx, KC_ATTEND_DECODE, st);
-    e = launch_pdl(attend_decode_kernel<D, G>, dim3(nsplit, p.HG, B), dim3(DEC_WARPS * 32), smem, st, p);
+    e = launch_pdl(attend_decode_kernel<D, G, TWO>, dim3(nsplit, p.HG, B), dim3(DEC_WARPS * 32), smem, st, p);
     ctx->launches += 1;
     return e;
 }
 
-template <int D>
+template <int D, bool TWO>
 static cudaError_t launch_decode(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
     switch (p.G) {
-        case 1: return launch_decode_t<D, 1>(ctx, p, B, n_att_max, st);
-        case 2: return launch_decode_t<D, 2>(ctx, p, B, n_att_max, st);
-        case 4: return launch_decode_t<D, 4>(ctx, p, B, n_att_max, st);
-        case 7: return launch_decode_t<D, 7>(ctx, p, B, n_att_max, st);
-        case 8: return launch_decode_t<D, 8>(ctx, p, B, n_att_max, st);
+        case 1: return launch_decode_t<D, 1, TWO>(ctx, p, B, n_att_max, st);
+        case 2: return launch_decode_t<D, 2, TWO>(ctx, p, B, n_att_max, st);
+        case 4: return launch_decode_t<D, 4, TWO>(ctx, p, B, n_att_max, st);
+        case 7: return launch_decode_t<D, 7, TWO>(ctx, p, B, n_att_max, st);
+        case 8: return launch_decode_t<D, 8, TWO>(ctx, p, B, n_att_max, st);
     }
     return cudaErrorNotSupported;
 }
 
-template <int D, int NW, int BN>
+template <int D, int NW, int BN, bool TWO>
 static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
     constexpr int BM = NW * 16;
     const int R = p.l_C * p.G;
     const int row_tiles = (R + BM - 1) / BM;
-    constexpr int smem = (BM + 4 * BN) * (D / 8) * 16;
-    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    constexpr int smem = ((TWO ? 2 : 1) * BM + 4 * BN) * (D / 8) * 16;
+    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int nsplit = 1;
     if (R <= kAttSplitRows && row_tiles == 1) {
         // split the key list so that one wave of CTAs fills the machine (never a second, short wave)
         int per_sm = 1;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN>, NW * 32, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN, TWO>, NW * 32, smem);
         if (e != cudaSuccess) return e;
         const int ctas = p.HG * B;
         const int n_tiles = (n_att_max + BN - 1) / BN;
@@ -648,7 +708,7 @@ static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     p.nsplit = nsplit;
     {
         ProfScope prof(ctx, KC_ATTEND_SMALL, st);
-        attend_kernel<D, NW, BN><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
+        attend_kernel<D, NW, BN, TWO><<<dim3(row_tiles, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
     }
     ctx->launches += 1;
     if (nsplit > 1) {
@@ -659,11 +719,35 @@ static cudaError_t launch_attend_t(esa_ctx* ctx, AttendParams& p, int B, int n_a
     return cudaGetLastError();
 }
 
-cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* K,
-                          const __nv_bfloat16* V, const SeqMeta& meta, const int32_t* idx,
-                          const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st) {
+template <bool TWO>
+static cudaError_t launch_small(esa_ctx* ctx, AttendParams& p, int B, int l_C, int n_att_max, cudaStream_t st) {
+    const int R = l_C * ctx->G;
+    if (l_C == 1) {
+        // decode: streaming kernel for the usual group sizes
+        cudaError_t e = ctx->d == 128 ? launch_decode<128, TWO>(ctx, p, B, n_att_max, st)
+                                      : launch_decode<64, TWO>(ctx, p, B, n_att_max, st);
+        if (e != cudaErrorNotSupported) return e;
+    }
+    if (ctx->d == 128) {
+        if (R <= 16) return launch_attend_t<128, 1, 32, TWO>(ctx, p, B, n_att_max, st);
+        if (R <= 64) return launch_attend_t<128, 4, 64, TWO>(ctx, p, B, n_att_max, st);
+        return launch_attend_t<128, 8, 64, TWO>(ctx, p, B, n_att_max, st);
+    } else if (ctx->d == 64) {
+        if (R <= 16) return launch_attend_t<64, 1, 32, TWO>(ctx, p, B, n_att_max, st);
+        if (R <= 64) return launch_attend_t<64, 4, 64, TWO>(ctx, p, B, n_att_max, st);
+        return launch_attend_t<64, 8, 64, TWO>(ctx, p, B, n_att_max, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// Qg / Kg: queries and key cache used against I and M_k (Section 3.2); null = Q / K.
+cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
+                          const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
+                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st) {
+    const bool two = (Qg && Qg != Q) || (Kg && Kg != K);
     AttendParams p;
-    p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
+    p.Q = Q; p.K = K; p.Qg = Qg ? Qg : Q; p.Kg = Kg ? Kg : K;
+    p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
     p.status = ctx->status;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
@@ -679,24 +763,10 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
     if (R > kAttSplitRows) {
         // prefill-sized chunks: tcgen05 kernel (a split key list is merged inside it)
         int nsplit = 1;
-        return launch_attend_tc(ctx, B, l_C, Q, K, V, meta, idx, n_sel, O, n_att_max, st, &nsplit);
+        return launch_attend_tc(ctx, B, l_C, Q, two ? p.Qg : nullptr, K, two ? p.Kg : nullptr, V, meta, idx, n_sel, O, n_att_max, st,
+                                &nsplit);
     }
-    if (l_C == 1) {
-        // decode: streaming kernel for the usual group sizes
-        cudaError_t e = ctx->d == 128 ? launch_decode<128>(ctx, p, B, n_att_max, st)
-                                      : launch_decode<64>(ctx, p, B, n_att_max, st);
-        if (e != cudaErrorNotSupported) return e;
-    }
-    if (ctx->d == 128) {
-        if (R <= 16) return launch_attend_t<128, 1, 32>(ctx, p, B, n_att_max, st);
-        if (R <= 64) return launch_attend_t<128, 4, 64>(ctx, p, B, n_att_max, st);
-        return launch_attend_t<128, 8, 64>(ctx, p, B, n_att_max, st);
-    } else if (ctx->d == 64) {
-        if (R <= 16) return launch_attend_t<64, 1, 32>(ctx, p, B, n_att_max, st);
-        if (R <= 64) return launch_attend_t<64, 4, 64>(ctx, p, B, n_att_max, st);
-        return launch_attend_t<64, 8, 64>(ctx, p, B, n_att_max, st);
-    }
-    return cudaErrorInvalidValue;
+    return two ? launch_small<true>(ctx, p, B, l_C, n_att_max, st) : launch_small<false>(ctx, p, B, l_C, n_att_max, st);
 }
 
 // ---------------------------------------------------------------------------
@@ -726,10 +796,10 @@ template <int D, int NW, int BN>
 cudaError_t launch_noalloc_t(const NoAllocDevice& dev, AttendParams& p, int B, int n_att_max, cudaStream_t st) {
     const int R = p.l_C * p.G;
     constexpr int smem = (NW * 16 + 4 * BN) * (D / 8) * 16;
-    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(attend_kernel<D, NW, BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int per_sm = 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN>, NW * 32, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attend_kernel<D, NW, BN, false>, NW * 32, smem);
     if (e != cudaSuccess) return e;
     const int n_tiles = (n_att_max + BN - 1) / BN;
     int nsplit = (per_sm * dev.num_sms) / (p.HG * B);
@@ -738,7 +808,7 @@ cudaError_t launch_noalloc_t(const NoAllocDevice& dev, AttendParams& p, int B, i
     while (nsplit > 1 && (size_t)B * p.HG * nsplit * R * (D + 2) > kNoAllocPartFloats) --nsplit;
     if (nsplit < 1) nsplit = 1;
     p.nsplit = nsplit;
-    attend_kernel<D, NW, BN><<<dim3(1, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
+    attend_kernel<D, NW, BN, false><<<dim3(1, p.HG, B * nsplit), NW * 32, smem, st>>>(p);
     if (nsplit > 1) attend_merge_kernel<D><<<dim3((R + 7) / 8, p.HG, B), 256, 0, st>>>(p);
     return cudaGetLastError();
 }
@@ -804,6 +874,7 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
 
     AttendParams p;
     p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
+    p.Qg = p.Q; p.Kg = p.K;
     p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr;
     p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
     p.top_k = cfg->top_k; p.nsplit = 1;

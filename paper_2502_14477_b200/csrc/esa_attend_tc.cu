@@ -63,6 +63,8 @@ constexpr float kRescaleThreshold = 8.0f;    // log2 domain
 struct TcAttendParams {
     const __nv_bfloat16* Q;
     const __nv_bfloat16* K;
+    const __nv_bfloat16* Qg;   // two-position attention (Section 3.2): queries / keys used against I and M_k
+    const __nv_bfloat16* Kg;
     const __nv_bfloat16* V;
     __nv_bfloat16* O;
     const int32_t* idx;
@@ -146,9 +148,14 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
     return r;
 }
 
-template <int D>
+// TWO (two-position attention): the list entries of I and M_k take their logits from Qg and Kg, the
+// entries of L and C from Q and K.  Both pairs of Q tiles stay in shared memory (three K/V stages instead
+// of four make room), the I u M_k part of the key list is padded to whole tiles so that a tile never
+// mixes the two, and the issuing warp picks the Q tiles by the tile's part.
+template <int D, bool TWO>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
+attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap qgmap, TcAttendParams p) {
+    constexpr int STAGES = TWO ? 3 : TC_STAGES;
     constexpr int CH = D / 8;                   // 16-byte chunks per row
     constexpr int Q_TILE_BYTES = 128 * D * 2;   // one 128-row Q tile
     constexpr int Q_BLK_BYTES = 128 * 128;      // one 64-column block of it
@@ -158,8 +165,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                               // 2 Q tiles
-    uint8_t* sK = sQ + 2 * Q_TILE_BYTES;              // TC_STAGES tiles
-    uint8_t* sV = sK + TC_STAGES * KV_TILE_BYTES;     // TC_STAGES tiles
+    uint8_t* sQg = sQ + 2 * Q_TILE_BYTES;             // 2 more (TWO)
+    uint8_t* sK = sQg + (TWO ? 2 * Q_TILE_BYTES : 0); // STAGES tiles
+    uint8_t* sV = sK + STAGES * KV_TILE_BYTES;        // STAGES tiles
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -180,11 +188,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
     if (tid == 0) {
         abort_flag = 0;
         mbar_init(bar(BAR_Q_FULL), p.q_tma ? 1 : TC_PRODUCERS);
-        for (int s = 0; s < TC_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_K_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_V_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_K_EMPTY + s), 2);          // one commit per Q tile's issuing warp
             mbar_init(bar(BAR_V_EMPTY + s), 2);
+        }
+        for (int s = 0; s < 4; ++s) {                    // [Q tile][buffer]
             mbar_init(bar(BAR_S_READY + s), 1);
             mbar_init(bar(BAR_P_READY + s), 128);        // every softmax thread of the tile arrives
         }
@@ -212,7 +222,12 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
 
     const int r_last = min(R, row0 + TC_ROWS) - 1;
     const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
-    const int n_tiles_all = (j_end + TC_BN - 1) / TC_BN;
+    // tiles: the first far_tiles cover the list entries [0, far_end) of I and M_k (TWO: padded to whole tiles),
+    // the rest the entries from far_end on
+    const int far_end = TWO ? n_glob : 0;
+    const int far_tiles = TWO ? (n_glob + TC_BN - 1) / TC_BN : 0;
+    auto tile_key0 = [&](int T) { return T < far_tiles ? T * TC_BN : far_end + (T - far_tiles) * TC_BN; };
+    const int n_tiles_all = far_tiles + max(0, (j_end - far_end + TC_BN - 1) / TC_BN);
     const int per = (n_tiles_all + p.nsplit - 1) / p.nsplit;
     const int tile_begin = split * per;
     const int tile_end = min(n_tiles_all, tile_begin + per);
@@ -234,11 +249,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
         float m_run = -INFINITY, l_run = 0.f;
 
         for (int j = 0; j < n_tiles; ++j) {
-            const int key0 = (tile_begin + j) * TC_BN;
+            const int key0 = tile_key0(tile_begin + j);
+            const bool far = tile_begin + j < far_tiles;
+            const int lim_t = far ? far_end : lim;           // first masked list position of this tile for this row
             const int u = j & 1;
             mbar_wait(bar(BAR_S_READY + qt * 2 + u), (j >> 1) & 1, wc);
             tc_fence_after_sync();
-            const bool need_mask = key0 + TC_BN > lim_min;
+            const bool need_mask = key0 + TC_BN > (far ? far_end : lim_min);
             // the score row of this thread: 64 fp32 columns
             uint32_t v[TC_BN];
             tmem_ld32(tS + u * 64, v);
@@ -247,7 +264,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             if (need_mask) {
 #pragma unroll
                 for (int i = 0; i < TC_BN; ++i)
-                    if (key0 + i >= lim) v[i] = 0xff800000u;     // -inf
+                    if (key0 + i >= lim_t) v[i] = 0xff800000u;   // -inf
             }
             float mxc[8];
 #pragma unroll
@@ -408,7 +425,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 // their O_READY before the arrival barrier above, so no MMA reads them any more.
                 const int64_t own_off = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;     // this lane's row of O, in elements
                 const uint32_t own_lo = (uint32_t)own_off, own_hi = (uint32_t)(own_off >> 32);
-                float4* ring = reinterpret_cast<float4*>(sK + warp_u * (2 * TC_STAGES * KV_TILE_BYTES / 8));
+                // (TWO: the ring starts at the second pair of Q tiles, idle as well, since three K/V stages alone are too small)
+                constexpr int RING_BYTES = (TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES;
+                static_assert(RING_BYTES / 8 >= 2 * 32 * (D / 8) * 16, "two buffers of 32 rows x D/2 floats per warp");
+                float4* ring = reinterpret_cast<float4*>((TWO ? sQg : sK) + warp_u * (RING_BYTES / 8));
                 const int n_other = p.nsplit - 1, n_pairs = 2 * n_other;
                 auto other = [&](int i) { const int s = i % n_other; return s + (s >= split ? 1 : 0); };
                 auto issue = [&](int i) {
@@ -533,13 +553,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
         if (n_tiles > 0 && p.q_tma) {
             // two boxes per 64-column block: rows (query, head-in-group) of one key/value head
             if (ptid == 0) {
-                mbar_arrive_expect_tx(bar(BAR_Q_FULL), 2 * Q_TILE_BYTES);
+                mbar_arrive_expect_tx(bar(BAR_Q_FULL), (TWO ? 4 : 2) * Q_TILE_BYTES);
 #pragma unroll
                 for (int qt = 0; qt < 2; ++qt)
 #pragma unroll
-                    for (int blk = 0; blk < D / 64; ++blk)
+                    for (int blk = 0; blk < D / 64; ++blk) {
                         tma_load_3d(smem_u32(sQ + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), &qmap, blk * 64, kvh * G,
                                     b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
+                        if (TWO)
+                            tma_load_3d(smem_u32(sQg + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), &qgmap, blk * 64, kvh * G,
+                                        b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
+                    }
             }
         } else if (n_tiles > 0) {
             // group sizes that do not divide 128: 16-byte copies, row by row
@@ -547,34 +571,40 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
                 const int row = row0 + r;
                 const bool ok = row < R;
                 const int cq = ok ? row / G : 0, g = ok ? row % G : 0;
-                const __nv_bfloat16* src = p.Q + (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + chunk * 8;
+                const int64_t qoff = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + chunk * 8;
                 const int rr = r & 127;
-                uint8_t* dst = sQ + (r >> 7) * Q_TILE_BYTES + (chunk >> 3) * Q_BLK_BYTES + rr * 128 + ((cin ^ (rr & 7)) << 4);
-                cp_async16(dst, src, ok ? 16 : 0);
+                const uint32_t doff = (r >> 7) * Q_TILE_BYTES + (chunk >> 3) * Q_BLK_BYTES + rr * 128 + ((cin ^ (rr & 7)) << 4);
+                cp_async16(sQ + doff, p.Q + qoff, ok ? 16 : 0);
+                if (TWO) cp_async16(sQg + doff, p.Qg + qoff, ok ? 16 : 0);
             }
             cp_async_arrive_noinc(bar(BAR_Q_FULL));
         }
         const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
+        const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
         const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
         const uint32_t blk_off = (chunk >> 3) * KV_BLK_BYTES;
         int bad_idx = 0;
         for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % TC_STAGES;
-            const uint32_t ph = ((j / TC_STAGES) & 1) ^ 1;
-            const int key0 = (tile_begin + j) * TC_BN;
+            const int s = j % STAGES;
+            const uint32_t ph = ((j / STAGES) & 1) ^ 1;
+            const int key0 = tile_key0(tile_begin + j);
+            const bool far = tile_begin + j < far_tiles;
+            const int row_lim = far ? far_end : n_att;      // list positions of this tile end here
+            const __nv_bfloat16* Ksrc = far ? Kgb : Kb;
             int pos[TC_BN / RSTEP];
             uint32_t from_idx = 0;                      // rows whose position was read from the selection
 #pragma unroll
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int jj = key0 + rsub + it * RSTEP;
                 int q = -1;
-                if (jj < i_end) q = jj;
+                if (jj >= row_lim) q = -1;
+                else if (jj < i_end) q = jj;
                 else if (jj < n_glob) {
                     q = __ldg(idx + (jj - i_end));
                     from_idx |= 1u << it;
-                } else if (jj < n_att) q = m_end + (jj - n_glob);
+                } else q = m_end + (jj - n_glob);
                 pos[it] = q;
             }
             mbar_wait(bar(BAR_K_EMPTY + s), ph, wc);
@@ -587,7 +617,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             for (int it = 0; it < TC_BN / RSTEP; ++it) {
                 const int r = rsub + it * RSTEP;
                 uint8_t* dst = sK + s * KV_TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
-                cp_async16(dst, Kb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
+                cp_async16(dst, Ksrc + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
             }
             cp_async_arrive_noinc(bar(BAR_K_FULL + s));
             mbar_wait(bar(BAR_V_EMPTY + s), ph, wc);
@@ -612,14 +642,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
         constexpr uint32_t ID_PV = idesc_bf16(128, D, false, true);
         const uint32_t hi = desc_hi_sw128();
         const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)) + qt * (Q_TILE_BYTES >> 4);
+        const uint32_t qglo = desc_lo_kmajor(smem_u32(sQg)) + qt * (Q_TILE_BYTES >> 4);
         const uint32_t klo = desc_lo_kmajor(smem_u32(sK)), vlo = desc_lo_mnmajor(smem_u32(sV), KV_BLK_BYTES);
         const uint32_t dS = tmem + qt * 128, dO = tmem + 256 + qt * D;
         // descriptor low words advance by compile-time constants (bytes >> 4)
-        auto issue_qk = [&](int s, int u) {                 // S[u] = Q . K[s]^T
+        auto issue_qk = [&](int s, int u, int j) {          // S[u] = Q . K[s]^T for the CTA's j-th tile
             const uint32_t b0 = klo + s * (KV_TILE_BYTES >> 4);
+            const uint32_t qsel = (TWO && tile_begin + j < far_tiles) ? qglo : qlo;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
-                umma_ss(dS + u * 64, qlo + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
+                umma_ss(dS + u * 64, qsel + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
                         b0 + (((ks >> 2) * KV_BLK_BYTES + (ks & 3) * 32) >> 4), hi, ID_QK, ks, lead);
         };
         auto issue_pv = [&](int s, int u, int acc) {         // O (+)= P[u] . V[s]
@@ -633,16 +665,16 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             mbar_wait(bar(BAR_K_FULL + j), 0, wc);
             fence_async_smem();
             tc_fence_after_sync();
-            issue_qk(j, j);
+            issue_qk(j, j, j);
             umma_commit(bar(BAR_S_READY + qt * 2 + j), lead);
             umma_commit(bar(BAR_K_EMPTY + j), lead);
         }
         for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % TC_STAGES, u = j & 1;
-            const int jn = j + 2, sn = jn % TC_STAGES;
+            const int s = j % STAGES, u = j & 1;
+            const int jn = j + 2, sn = jn % STAGES;
             const bool more = jn < n_tiles;
-            mbar_wait(bar(BAR_V_FULL + s), (j / TC_STAGES) & 1, wc);
-            if (more) mbar_wait(bar(BAR_K_FULL + sn), (jn / TC_STAGES) & 1, wc);
+            mbar_wait(bar(BAR_V_FULL + s), (j / STAGES) & 1, wc);
+            if (more) mbar_wait(bar(BAR_K_FULL + sn), (jn / STAGES) & 1, wc);
             fence_async_smem();
             mbar_wait(bar(BAR_P_READY + qt * 2 + u), (j >> 1) & 1, wc);
             tc_fence_after_sync();
@@ -651,7 +683,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
             if (j + 1 == n_tiles) umma_commit(bar(BAR_O_READY + qt), lead);
             umma_commit(bar(BAR_V_EMPTY + s), lead);
             if (more) {
-                issue_qk(sn, u);              // reuses buffer u after the P V product above, in issue order
+                issue_qk(sn, u, jn);          // reuses buffer u after the P V product above, in issue order
                 umma_commit(bar(BAR_S_READY + qt * 2 + u), lead);
                 umma_commit(bar(BAR_K_EMPTY + sn), lead);
             }
@@ -665,20 +697,20 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, TcAttendParams p) {
 
 }  // namespace
 
-template <int D>
+template <int D, bool TWO>
 static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_max, cudaStream_t st, int* nsplit_out) {
     const int R = p.l_C * p.G;
     const int row_tiles = (R + TC_ROWS - 1) / TC_ROWS;
     p.Rp = (R + 1) & ~1;
     if ((size_t)B * p.HG * row_tiles > ctx->att_count_elems) return cudaErrorNotSupported;
-    constexpr int smem = 2 * 128 * D * 2 + 2 * TC_STAGES * TC_BN * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    constexpr int smem = (TWO ? 4 : 2) * 128 * D * 2 + 2 * (TWO ? 3 : TC_STAGES) * TC_BN * D * 2 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     // the in-kernel register split assumes the launch allocation it was sized for
     static int regs_checked = 0;
     if (!regs_checked) {
         cudaFuncAttributes fa;
-        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D>);
+        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D, TWO>);
         if (e != cudaSuccess) return e;
         if (fa.numRegs != TC_REGS_LAUNCH) return cudaErrorInvalidConfiguration;
         regs_checked = 1;
@@ -686,7 +718,7 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     // Split the key list when that fills the machine better: cost model = waves x tiles per CTA
     // (+1 tile-equivalent of fixed work per CTA), one CTA per SM.
     const int ctas = row_tiles * p.HG * B;
-    const int n_tiles = (n_att_max + TC_BN - 1) / TC_BN;
+    const int n_tiles = (n_att_max + TC_BN - 1) / TC_BN + (TWO ? 1 : 0);
     int best = 1;
     double best_cost = 1e30;
     for (int ns = 1; ns <= kAttPrefillSplits && ns <= n_tiles; ++ns) {
@@ -698,29 +730,34 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     }
     p.nsplit = best;
     *nsplit_out = best;
-    CUtensorMap qmap;
+    CUtensorMap qmap, qgmap;
     p.q_tma = make_tensor_map_q(&qmap, p.Q, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
+    if (p.q_tma && TWO) p.q_tma = make_tensor_map_q(&qgmap, p.Qg, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
     if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
+    if (!p.q_tma || !TWO) memset(&qgmap, 0, sizeof(qgmap));
     ProfScope prof(ctx, KC_ATTEND_TC, st);
-    e = launch_pdl(attend_tc_kernel<D>, dim3(row_tiles, p.HG, B * best), dim3(TC_THREADS), smem, st, qmap, p);
+    e = launch_pdl(attend_tc_kernel<D, TWO>, dim3(row_tiles, p.HG, B * best), dim3(TC_THREADS), smem, st, qmap, qgmap, p);
     ctx->launches += 1;
     return e;
 }
 
 // Returns cudaErrorNotSupported when this path does not cover the shape (the caller then
 // uses the split kernel); nsplit_out reports how many ways the key list was split (merged in-kernel).
-cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* K,
-                             const __nv_bfloat16* V, const SeqMeta& meta, const int32_t* idx, const int32_t* n_sel,
-                             __nv_bfloat16* O, int n_att_max, cudaStream_t st, int* nsplit_out) {
+cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
+                             const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
+                             const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, int n_att_max, cudaStream_t st,
+                             int* nsplit_out) {
+    const bool two = Qg != nullptr || Kg != nullptr;
     TcAttendParams p;
-    p.Q = Q; p.K = K; p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.status = ctx->status;
+    p.Q = Q; p.K = K; p.Qg = Qg ? Qg : Q; p.Kg = Kg ? Kg : K;
+    p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.status = ctx->status;
     p.unit_count = ctx->att_count;
     p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
     p.meta = meta;
-    if (ctx->d == 128) return launch_tc<128>(ctx, p, B, n_att_max, st, nsplit_out);
-    if (ctx->d == 64) return launch_tc<64>(ctx, p, B, n_att_max, st, nsplit_out);
+    if (ctx->d == 128) return two ? launch_tc<128, true>(ctx, p, B, n_att_max, st, nsplit_out) : launch_tc<128, false>(ctx, p, B, n_att_max, st, nsplit_out);
+    if (ctx->d == 64) return two ? launch_tc<64, true>(ctx, p, B, n_att_max, st, nsplit_out) : launch_tc<64, false>(ctx, p, B, n_att_max, st, nsplit_out);
     return cudaErrorNotSupported;
 }
 

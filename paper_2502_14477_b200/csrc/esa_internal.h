@@ -154,15 +154,16 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
 cudaError_t launch_select_all(esa_ctx* ctx, int B, const SeqMeta& meta, int32_t* idx_out,
                               int32_t* n_sel_out, cudaStream_t st);
 
-cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
-                          const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
-                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
-                          cudaStream_t st);
+// Qg / Kg: queries and key cache used against I and M_k (two-position attention, Section 3.2); null = Q / K.
+cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
+                          const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
+                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st);
 
 // Prefill-sized chunks (l_C * H/H_G > kAttSplitRows) on tcgen05; *nsplit_out reports the number of
 // key-list splits (their partials pass through ctx->att_part and are merged inside the kernel).
-cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q,
-                             const __nv_bfloat16* K, const __nv_bfloat16* V, const SeqMeta& meta,
+// Qg / Kg non-null: two-position attention (both given then).
+cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
+                             const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
                              const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
                              int n_att_max, cudaStream_t st, int* nsplit_out);
 

@@ -397,6 +397,64 @@ def test_compress_keys_on_a_side_stream_matches_the_serial_order():
         assert torch.equal(i0[0, :k], i1[0, :k])
 
 
+# ------------------------------------------------ two-position attention (Section 3.2)
+def _two_position_case(cfg, t, l_C, heads=None, use_qfar=True, use_kfar=True, n_sel=None, seed=0):
+    """esa_attend_two_position against the oracle: I and M_k attended with a second encoding of the
+    queries and keys (stand-ins: independent seeded tensors), L and C with the first."""
+    p = hp.oracle_params(cfg)
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=1)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, B=1)
+    seq.fill_kv(0, n)
+    Qb = syn.qkv_rows(cfg, "q", t, n)
+    Qfb = syn.qkv_rows(cfg, "q", t, n, layer=7)              # the far-position encoding of the same tokens
+    Kfb = syn.qkv_rows(cfg, "k", 0, n, layer=7)
+    Q, Qf = hp.bits_to_torch(Qb)[None].contiguous(), hp.bits_to_torch(Qfb)[None].contiguous()
+    Kf = hp.bits_to_torch(Kfb)[None].contiguous()
+    i_end, m_end = orc.partition(t, cfg.l_I, cfg.l_L)
+    l_M = m_end - i_end
+    kk = min(cfg.k, l_M) if n_sel is None else n_sel
+    g = np.random.default_rng(seed)
+    sel = np.sort(g.choice(np.arange(i_end, m_end), size=kk, replace=False)) if kk else np.zeros(0, np.int64)
+    seq.idx[0, :kk] = torch.from_numpy(sel.astype(np.int32)).cuda()
+    seq.n_sel[0] = kk
+    O = torch.full_like(Q, float("nan"))
+    ctx.attend_two_position(Q, Qf if use_qfar else None, seq.K, Kf if use_kfar else None, seq.V, [t], seq.idx, seq.n_sel, O,
+                            sync=True)
+    assert ctx.last_device_status() == 0
+    want = orc.attend(syn.bf16_bits_to_f64(Qb), hp.torch_to_f64(seq.K[0]), hp.torch_to_f64(seq.V[0]), sel, t, p, heads=heads,
+                      Q_global=syn.bf16_bits_to_f64(Qfb) if use_qfar else None,
+                      K_global=syn.bf16_bits_to_f64(Kfb) if use_kfar else None)
+    hp.check_attention(O[0], want, what=f"two-position {cfg.name} t={t} l_C={l_C}", heads=heads)
+    # the far tensors matter: where I and M_k are a fair share of the list, the one-position result differs
+    if (use_qfar or use_kfar) and 4 * (i_end + kk) >= n - m_end:
+        one = orc.attend(syn.bf16_bits_to_f64(Qb), hp.torch_to_f64(seq.K[0]), hp.torch_to_f64(seq.V[0]), sel, t, p, heads=heads)
+        hs = heads if heads is not None else slice(None)
+        assert np.abs(one[:, hs] - want[:, hs]).max() > 2 * hp.ATT_MAX_ABS
+
+
+@pytest.mark.parametrize("t,l_C", [(3968, 128), (3000, 77), (4100, 1), (2000, 5), (640, 128), (0, 128), (300, 1)])
+def test_two_position_attention_c1(t, l_C):
+    _two_position_case(syn.get_config("c1"), t, l_C)
+
+
+def test_two_position_attention_partial_tensors_and_ragged_far_part():
+    cfg = syn.get_config("c1")
+    _two_position_case(cfg, 3968, 128, use_kfar=False)                 # far queries only
+    _two_position_case(cfg, 3968, 128, use_qfar=False)                 # far keys only
+    _two_position_case(cfg, 3968, 128, n_sel=201)                      # |I| + |M_k| = 205: the far part ends inside a tile
+    _two_position_case(cfg, 4100, 1, n_sel=201)
+    _two_position_case(cfg, 4000, 9, n_sel=37)
+
+
+def test_two_position_attention_llama_shape_and_group_of_seven():
+    _two_position_case(syn.get_config("c2"), 16 * 512, 512, heads=[0, 5, 31])
+    _two_position_case(syn.get_config("c2"), 9000, 1)
+    cfg = syn.get_config("c4").with_(S=16384, l_C=256, l_L=1024, k=1024)
+    _two_position_case(cfg, 40 * 256, 256, heads=[0, 6, 7, 27])
+    _two_position_case(cfg, 10000, 1)
+
+
 # ------------------------------------------------------- device-side safety nets
 @pytest.mark.parametrize("t,l_C", [(3000, 1), (3000, 5), (2944, 128)])
 def test_selected_position_outside_M_is_clamped_and_reported(t, l_C):

@@ -277,15 +277,70 @@ def test_attend_subset_matches_library_with_explicit_mask():
     assert np.allclose(got, sdpa_ref(Q, K, V, vis, 0.37), rtol=1e-10, atol=1e-12)
 
 
-def test_alg1_two_part_merge_equals_single_softmax():
+def test_attention_by_parts_equals_single_softmax():
+    """Algorithm 1: a causal part on [L, C] and a non-causal part on [I, M_k], merged by the
+    softmax of their log-normalisers, equal one softmax over the union; so does any other cut."""
     g = rng(14)
     t, l_C, H, H_G, d = 80, 7, 4, 1, 8
     Q, K, V = make_qkv(g, t, l_C, H, H_G, d)
-    Q *= 4.0                                        # spread the two lse values apart
+    Q *= 4.0                                        # spread the two log-normalisers apart
     p = orc.EsaParams(l_I=5, l_L=16, k=9, eps=1)
     i_end, m_end = orc.partition(t, p.l_I, p.l_L)
     sel = np.sort(g.choice(np.arange(i_end, m_end), size=9, replace=False))
-    assert np.allclose(orc.attend(Q, K, V, sel, t, p), orc.attend_alg1(Q, K, V, sel, t, p), rtol=1e-10, atol=1e-12)
+    want = orc.attend(Q, K, V, sel, t, p)
+    assert np.allclose(want, orc.attend_by_parts(Q, K, V, sel, t, p), rtol=1e-10, atol=1e-12)
+    assert np.allclose(want, orc.attend_by_parts(Q, K, V, sel, t, p, cuts=[3, 20, 33]), rtol=1e-10, atol=1e-12)
+    # no far keys at all (chunk 0): the near part alone
+    Q0, K0, V0 = make_qkv(g, 0, l_C, H, H_G, d)
+    assert np.allclose(orc.attend(Q0, K0, V0, np.zeros(0, np.int64), 0, p),
+                       orc.attend_by_parts(Q0, K0, V0, np.zeros(0, np.int64), 0, p), rtol=1e-10, atol=1e-12)
+
+
+def test_merge_weights_are_the_normalised_exponentials_of_the_log_normalisers():
+    """The merge weights written out without the max subtraction (safe here: small values)."""
+    g = rng(21)
+    o1, o2 = g.standard_normal((5, 3)), g.standard_normal((5, 3))
+    l1, l2 = g.standard_normal(5), g.standard_normal(5)
+    se = np.exp(np.stack([l1, l2]))
+    fac = se / se.sum(axis=0)
+    want = o1 * fac[0][:, None] + o2 * fac[1][:, None]
+    assert np.allclose(orc.merge_softmax_parts([(o1, l1), (o2, l2)]), want, rtol=1e-12, atol=1e-14)
+    # an empty part (log-normaliser -inf) carries no weight
+    assert np.allclose(orc.merge_softmax_parts([(o1, l1), (o2, np.full(5, -np.inf))]), o1)
+
+
+def test_two_position_attention_bruteforce():
+    """Section 3.2 / Algorithm 1 with distinct tensors: far-position queries and keys for
+    [I, M_k], near-position ones for [L, C], checked against explicit loops (two softmax
+    normalisers per row and the merge), and against ``attend`` with the same arguments."""
+    g = rng(22)
+    t, l_C, H, H_G, d = 40, 5, 4, 2, 8
+    Q, K, V = make_qkv(g, t, l_C, H, H_G, d)
+    Qg = rand_bf16(g, l_C, H, d)
+    Kg = rand_bf16(g, t + l_C, H_G, d)
+    p = orc.EsaParams(l_I=3, l_L=9, k=6, eps=0)
+    i_end, m_end = orc.partition(t, p.l_I, p.l_L)
+    sel = np.sort(g.choice(np.arange(i_end, m_end), size=6, replace=False))
+    scale = 1.0 / math.sqrt(d)
+    far = list(range(i_end)) + sel.tolist()
+    want = np.zeros((l_C, H, d))
+    for c in range(l_C):
+        near = list(range(m_end, t + c + 1))
+        for h in range(H):
+            kv = h // (H // H_G)
+            lf = [scale * float(Qg[c, h] @ Kg[j, kv]) for j in far]
+            ln = [scale * float(Q[c, h] @ K[j, kv]) for j in near]
+            zf, zn = sum(math.exp(x) for x in lf), sum(math.exp(x) for x in ln)
+            of = sum(math.exp(x) * V[j, kv] for x, j in zip(lf, far)) / zf
+            on = sum(math.exp(x) * V[j, kv] for x, j in zip(ln, near)) / zn
+            want[c, h] = (zf * of + zn * on) / (zf + zn)
+    got = orc.attend(Q, K, V, sel, t, p, Q_global=Qg, K_global=Kg)
+    assert np.allclose(got, want, rtol=1e-10, atol=1e-12)
+    assert np.allclose(orc.attend_by_parts(Q, K, V, sel, t, p, Q_global=Qg, K_global=Kg), want, rtol=1e-10, atol=1e-12)
+    # identical tensors for both positions give the one-position result
+    assert np.allclose(orc.attend(Q, K, V, sel, t, p, Q_global=Q, K_global=K), orc.attend(Q, K, V, sel, t, p))
+    # and a different far query really changes the output
+    assert not np.allclose(got, orc.attend(Q, K, V, sel, t, p))
 
 
 def test_every_initial_local_and_current_key_is_attended():
