@@ -130,6 +130,22 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
                             const void* kc_cache, const int64_t* n_prev,
                             int32_t* idx_out, int32_t* n_sel_out, void* stream);
 
+/* Selection on full-dimension scores, the two variants the paper compares the compressed
+ * scores with (no compressors involved; K_cache is read instead of the compressed-key cache):
+ *   ESA_SCORE_UNIFORM   Eq. 3: f_s(m; c) = sum over the H heads of q_{h,c} . k_{h,m}, then Eq. 4, 8, 2
+ *                       ("uniform" in Section 4.3: the method without dimensionality reduction; its
+ *                       selection is the ground truth of the recall measurement of Fig. 3)
+ *   ESA_SCORE_PER_HEAD  Section 4.3 "individual": Eq. 4 per head, a token's score is the largest of
+ *                       its H head scores; then Eq. 8 and Eq. 2
+ * Q_cur: device [B, l_C, H, d]; K_cache: device [B, max_tokens, H_G, d] (rows of M are read).
+ * Outputs as for esa_select.  bf16 products, fp32 accumulation over all heads and dimensions. */
+typedef enum { ESA_SCORE_UNIFORM = 0, ESA_SCORE_PER_HEAD = 1 } esa_score_mode;
+esa_status esa_select_full(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                           const int64_t* n_prev, int32_t mode, int32_t* idx_out, int32_t* n_sel_out);
+esa_status esa_select_full_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                                 const int64_t* n_prev, int32_t mode, int32_t* idx_out, int32_t* n_sel_out,
+                                 void* stream);
+
 /* Eq. 1 / Algorithm 1.  Q_cur: device [B, l_C, H, d].  K_cache, V_cache: device
  * [B, max_tokens, H_G, d] that already hold C at rows [n_prev[b], n_prev[b]+l_C).
  * idx: device int32 [B, top_k] and n_sel: device int32 [B] as written by esa_select

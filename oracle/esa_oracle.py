@@ -145,6 +145,52 @@ def select(qc: np.ndarray, kc_M: np.ndarray, k: int, eps: int):
 
 
 # ----------------------------------------------------------------------------
+# Eq. 3 and Section 4.3: scores without dimensionality reduction
+# ----------------------------------------------------------------------------
+def scores_full(Q_C: np.ndarray, K_M: np.ndarray) -> np.ndarray:
+    """Eq. 3: f_s(m; c) = sum over the H query heads of q_{h,c} . k_{h,m}, where head h reads
+    key/value head h // (H/H_G).  Q_C [l_C,H,d], K_M [l_M,H_G,d] -> fp32 [l_C, l_M]."""
+    Q_C, K_M = np.asarray(Q_C, np.float64), np.asarray(K_M, np.float64)
+    H, g = Q_C.shape[1], Q_C.shape[1] // K_M.shape[1]
+    S = np.zeros((Q_C.shape[0], K_M.shape[0]), np.float64)
+    for h in range(H):
+        S += Q_C[:, h, :] @ K_M[:, h // g, :].T
+    return S.astype(np.float32)
+
+
+def aggregate_per_head(Q_C: np.ndarray, K_M: np.ndarray) -> np.ndarray:
+    """Section 4.3, "individual": every head scores the tokens by itself -- Eq. 4 on its own
+    logits q_{h,c} . k_{h,m} -- and a token's score is the largest of its H head scores."""
+    Q_C, K_M = np.asarray(Q_C, np.float64), np.asarray(K_M, np.float64)
+    H, g = Q_C.shape[1], Q_C.shape[1] // K_M.shape[1]
+    best = None
+    for h in range(H):
+        s_h = aggregate((Q_C[:, h, :] @ K_M[:, h // g, :].T).astype(np.float32))
+        best = s_h if best is None else np.maximum(best, s_h)
+    return best
+
+
+def select_full(Q_C: np.ndarray, K_M: np.ndarray, k: int, eps: int, per_head: bool = False):
+    """Selection on full-dimension scores: Eq. 3 -> Eq. 4 ("uniform", the paper's method without
+    compression) or the per-head vote, then Eq. 8 and Eq. 2 as usual.  Returns (indices into M,
+    pooled scores)."""
+    l_M = K_M.shape[0]
+    if l_M == 0:
+        return np.zeros(0, np.int64), np.zeros(0, np.float32)
+    s = aggregate_per_head(Q_C, K_M) if per_head else aggregate(scores_full(Q_C, K_M))
+    sp = proximity_pool(s, eps)
+    if k >= l_M:
+        return np.arange(l_M, dtype=np.int64), sp
+    return topk(sp, k), sp
+
+
+def recall(sel: np.ndarray, truth: np.ndarray) -> float:
+    """Share of the ground-truth selection that another selection also contains (Fig. 3)."""
+    truth = np.asarray(truth)
+    return float(np.isin(truth, np.asarray(sel)).mean()) if truth.size else 1.0
+
+
+# ----------------------------------------------------------------------------
 # Eq. 1 / Algorithm 1: attention over the reduced key set
 # ----------------------------------------------------------------------------
 def attend_positions(t: int, l_C: int, sel_abs: np.ndarray, p: EsaParams) -> np.ndarray:

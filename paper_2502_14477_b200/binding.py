@@ -78,6 +78,10 @@ _PROTOS = {
                              C.c_void_p, C.c_void_p]),
     "esa_select_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_select_full": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                  C.c_void_p, C.c_void_p]),
+    "esa_select_full_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_attend": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_attend_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
@@ -263,6 +267,25 @@ class Esa:
                                            _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_select")
+
+    def select_full(self, Q_cur, K_cache, n_prev, idx_out, n_sel_out, per_head=False, stream=None, sync=False):
+        """``esa_select_full``: selection on full-dimension scores (Eq. 3) or the per-head vote."""
+        c = self.cfg
+        B, l_C = Q_cur.shape[0], Q_cur.shape[1]
+        _check(Q_cur, "Q_cur", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        _check(K_cache, "K_cache", torch.bfloat16, (B, c.max_tokens, c.n_kv_heads, c.head_dim))
+        _check(idx_out, "idx_out", torch.int32, (B, c.top_k))
+        _check(n_sel_out, "n_sel_out", torch.int32, (B,))
+        npv = self._nprev(n_prev, B)
+        mode = 1 if per_head else 0
+        if sync:
+            st = self.lib.esa_select_full(self._h, B, _ptr(Q_cur), l_C, _ptr(K_cache), npv, mode, _ptr(idx_out),
+                                          _ptr(n_sel_out))
+        else:
+            st = self.lib.esa_select_full_async(self._h, B, _ptr(Q_cur), l_C, _ptr(K_cache), npv, mode, _ptr(idx_out),
+                                                _ptr(n_sel_out), _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_select_full")
 
     def attend(self, Q_cur, K_cache, V_cache, n_prev, idx, n_sel, O, stream=None, sync=False):
         c = self.cfg

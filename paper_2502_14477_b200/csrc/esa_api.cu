@@ -29,7 +29,7 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, rkey, skey, pkey, ghist0, cidx, slice_cnt, ticket, att, att_count, status, total;
+    size_t wq, wk, bq, bk, qc, rkey, rkey_heads, skey, pkey, ghist0, cidx, slice_cnt, ticket, att, att_count, status, total;
     size_t att_elems, att_count_elems, slice_stride;
 };
 
@@ -44,6 +44,7 @@ Layout make_layout(const esa_config* c) {
     L.bk = take(4 * c->d_c);
     L.qc = take(2 * (size_t)c->max_batch * c->max_chunk * c->d_c);
     L.rkey = take(4 * (size_t)c->max_batch * c->max_chunk);
+    L.rkey_heads = take(4 * (size_t)c->max_batch * c->max_chunk * c->n_q_heads);
     L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.ghist0 = take(4 * (size_t)c->max_batch * 2048);
@@ -165,6 +166,7 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->bk = reinterpret_cast<float*>(base + L.bk);
     c->Qc = reinterpret_cast<__nv_bfloat16*>(base + L.qc);
     c->rkey = reinterpret_cast<uint32_t*>(base + L.rkey);
+    c->rkey_heads = reinterpret_cast<uint32_t*>(base + L.rkey_heads);
     c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
     c->ghist0 = reinterpret_cast<uint32_t*>(base + L.ghist0);
@@ -349,8 +351,47 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
     e = launch_score(ctx, B, l_C, (const __nv_bfloat16*)kc_cache, smeta, max_lM, rkey_cleared, ghist_cleared, st,
                      &pooled_ready);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
-    e = launch_select(ctx, B, l_C, smeta, max_lM, pooled_ready, idx_out, n_sel_out, st);
+    e = launch_select(ctx, B, l_C == 1, smeta, max_lM, pooled_ready, idx_out, n_sel_out, st);
     return from_cuda(e);
+}
+
+esa_status esa_select_full_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                                 const int64_t* n_prev, int32_t mode, int32_t* idx_out, int32_t* n_sel_out, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!Q_cur || !K_cache || !n_prev || !idx_out || !n_sel_out || l_C <= 0) return ESA_ERR_INVALID_ARG;
+    if (mode != ESA_SCORE_UNIFORM && mode != ESA_SCORE_PER_HEAD) return ESA_ERR_INVALID_ARG;
+    if (l_C > ctx->cfg.max_chunk) return ESA_ERR_CAPACITY;
+    SeqMeta meta;
+    int max_lM = 0;
+    s = build_meta(ctx, B, n_prev, l_C, &meta, &max_lM);
+    if (s != ESA_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    bool any_small = false, any_large = false;
+    for (int b = 0; b < B; ++b) {
+        int lM = meta.m_end[b] - meta.i_end[b];
+        ctx->last_lM[b] = lM;
+        if (lM > ctx->cfg.top_k) any_large = true; else any_small = true;
+    }
+    ctx->last_scored = any_large;
+    ctx->last_q_rows = 0;
+    if (any_small && launch_select_all(ctx, B, meta, idx_out, n_sel_out, st) != cudaSuccess) return ESA_ERR_CUDA;
+    if (!any_large) return ESA_OK;
+    SeqMeta smeta = meta;
+    for (int b = 0; b < B; ++b)
+        if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
+    ctx->last_decode = false;
+    cudaError_t e = launch_score_full(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)K_cache, smeta, max_lM,
+                                      mode == ESA_SCORE_PER_HEAD, st);
+    if (e != cudaSuccess) return ESA_ERR_CUDA;
+    return from_cuda(launch_select(ctx, B, false, smeta, max_lM, false, idx_out, n_sel_out, st));
+}
+
+esa_status esa_select_full(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
+                           const int64_t* n_prev, int32_t mode, int32_t* idx_out, int32_t* n_sel_out) {
+    esa_status s = esa_select_full_async(ctx, B, Q_cur, l_C, K_cache, n_prev, mode, idx_out, n_sel_out, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
 }
 
 esa_status esa_select(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* kc_cache,
@@ -437,7 +478,8 @@ int32_t esa_kernel_class_count(void) { return KC_COUNT; }
 const char* esa_kernel_class_name(int32_t cls) {
     static const char* names[KC_COUNT] = {
         "compress_tc_kernel", "compress_gemv_kernel", "compress_kernel", "append_kv_kernel", "score_tc_kernel<.,1>",
-        "score_tc_kernel<.,2>", "score_pass_kernel<.,1>+<.,2>", "score_decode_kernel", "pool_hist_kernel",
+        "score_tc_kernel<.,2>", "score_pass_kernel<.,1>+<.,2>", "score_decode_kernel", "score_full_kernel<.,1>+<.,2>",
+        "pool_hist_kernel",
         "select_topk_kernel", "select_all_kernel", "attend_tc_kernel", "attend_decode_kernel", "attend_kernel",
         "attend_merge_kernel"};
     return cls >= 0 && cls < KC_COUNT ? names[cls] : "";

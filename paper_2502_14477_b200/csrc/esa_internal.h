@@ -45,7 +45,7 @@ struct RowMap {
 // Kernel classes of the per-kernel timing facility (esa_set_profiling / esa_read_profile).
 enum KernelClass {
     KC_COMPRESS_TC = 0, KC_COMPRESS_GEMV, KC_COMPRESS_MMA, KC_APPEND_KV, KC_SCORE_PASS1, KC_SCORE_PASS2, KC_SCORE_MMA,
-    KC_SCORE_DECODE, KC_POOL_HIST, KC_SELECT_TOPK, KC_SELECT_ALL, KC_ATTEND_TC, KC_ATTEND_DECODE, KC_ATTEND_SMALL,
+    KC_SCORE_DECODE, KC_SCORE_FULL, KC_POOL_HIST, KC_SELECT_TOPK, KC_SELECT_ALL, KC_ATTEND_TC, KC_ATTEND_DECODE, KC_ATTEND_SMALL,
     KC_ATTEND_MERGE, KC_COUNT
 };
 struct ProfRec {
@@ -71,6 +71,7 @@ struct esa_ctx {
     float* bk;           // [dc]
     __nv_bfloat16* Qc;   // [max_batch * max_chunk, dc]
     uint32_t* rkey;      // [max_batch * max_chunk] ordered keys of the row maxima r_c
+    uint32_t* rkey_heads;  // [max_batch, H, max_chunk] row maxima of the full-dimension / per-head scoring variants
     uint32_t* skey;      // [max_batch, max_tokens] unpooled aggregated scores (ordered keys) of the scoring paths that do not pool;
                          // afterwards the selection's candidate keys
     uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys (l_C = 1: of the pooled raw scores, r not yet subtracted)
@@ -145,9 +146,15 @@ cudaError_t launch_score(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_c
 cudaError_t launch_score_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* kc_cache,
                             const SeqMeta& meta, int max_lM, cudaStream_t st, bool* pooled_ready);
 
-// Eq. 8 (unless pooled_ready) + Eq. 2 -> idx_out / n_sel_out.
-cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, bool pooled_ready,
+// Eq. 8 (unless pooled_ready) + Eq. 2 -> idx_out / n_sel_out.  mapped: ctx->pkey holds the pooled RAW scores of a
+// single query per sequence and ctx->rkey[b] its maximum (the decode scoring kernel's output).
+cudaError_t launch_select(esa_ctx* ctx, int B, bool mapped, const SeqMeta& meta, int max_lM, bool pooled_ready,
                           int32_t* idx_out, int32_t* n_sel_out, cudaStream_t st);
+
+// Eq. 3 + Eq. 4 on the uncompressed queries and keys (per_head: the per-head vote of Section 4.3): unpooled keys to
+// ctx->skey, ctx->ghist0 zeroed.
+cudaError_t launch_score_full(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* K, const SeqMeta& meta,
+                              int max_lM, bool per_head, cudaStream_t st);
 
 // idx_out[b, 0..l_M) = i_end + 0..l_M-1, n_sel_out[b] = l_M for sequences with l_M <= top_k
 // (only_small = 1) or all sequences (only_small = 0).

@@ -479,7 +479,7 @@ __global__ void read_pooled_kernel(const uint32_t* __restrict__ pkey, const uint
 
 // pooled_ready: ctx->pkey / ctx->ghist0 already hold the pooled keys and their first-digit histogram;
 // otherwise ctx->skey holds unpooled keys and ctx->ghist0 is zero.
-cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int max_lM, bool pooled_ready,
+cudaError_t launch_select(esa_ctx* ctx, int B, bool mapped, const SeqMeta& meta, int max_lM, bool pooled_ready,
                           int32_t* idx_out, int32_t* n_sel_out, cudaStream_t st) {
     const int n_slices = (max_lM + SEL_SLICE - 1) / SEL_SLICE;
     if (n_slices < 1 || n_slices > ctx->sel_slice_stride) return cudaErrorInvalidConfiguration;
@@ -496,7 +496,7 @@ cudaError_t launch_select(esa_ctx* ctx, int B, int l_C, const SeqMeta& meta, int
     p.ckey = ctx->skey; p.cidx = ctx->cidx; p.slice_cnt = ctx->sel_slice_cnt; p.ticket = ctx->sel_ticket;
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.slice_stride = ctx->sel_slice_stride; p.top_k = ctx->cfg.top_k;
-    p.mapped = (l_C == 1) ? 1 : 0; p.l_C = l_C; p.meta = meta;
+    p.mapped = mapped ? 1 : 0; p.l_C = 1; p.meta = meta;     // (mapped mode reads rkey[b]: one query per sequence)
     constexpr size_t smem = (size_t)(SEL_MAX_SLICES_SMEM + 2 * SEL_STAGE_CAP) * 4;
     e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -397,6 +397,85 @@ def test_compress_keys_on_a_side_stream_matches_the_serial_order():
         assert torch.equal(i0[0, :k], i1[0, :k])
 
 
+# ------------------------------- full-dimension and per-head selection (Eq. 3, Section 4.3)
+class _FullResult:
+    """What check_index_sets reads, for a selection made on full-dimension scores."""
+
+    def __init__(self, sel_abs, pooled, rowmax, i_end, m_end):
+        self.sel_abs, self.pooled, self.rowmax, self.i_end, self.m_end = sel_abs, pooled, rowmax, i_end, m_end
+
+
+def _select_full_case(cfg, t, l_C, per_head, layer=0):
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=1, layer=layer)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, layer=layer, B=1)
+    seq.fill_kv(0, n)
+    Qb = syn.qkv_rows(cfg, "q", t, n, layer)
+    Q = hp.bits_to_torch(Qb)[None].contiguous()
+    Q64 = syn.bf16_bits_to_f64(Qb)
+    i_end, m_end = orc.partition(t, cfg.l_I, cfg.l_L)
+    K_M = hp.torch_to_f64(seq.K[0, i_end:m_end])
+    sel, sp = orc.select_full(Q64, K_M, cfg.k, cfg.eps, per_head=per_head)
+    ctx.select_full(Q, seq.K, [t], seq.idx, seq.n_sel, per_head=per_head, sync=True)
+    assert ctx.last_device_status() == 0
+    n_sel = int(seq.n_sel[0])
+    sel_gpu = seq.idx[0, :n_sel].cpu().numpy().astype(np.int64)
+    S_abs_max = float(np.abs(orc.scores_full(Q64, K_M)).max()) if m_end > i_end else 0.0
+    res = _FullResult(sel + i_end, sp, np.array([S_abs_max], np.float32), i_end, m_end)
+    hp.check_index_sets(sel_gpu, res, cfg.k, what=f"{cfg.name} full{'/per-head' if per_head else ''} t={t} l_C={l_C}")
+    if m_end - i_end > cfg.k:
+        # pooled scores within the fp32 accumulation bound of the d_H-long sums (the bound of the summed score
+        # also covers each head's own shorter sum)
+        K_rep = np.repeat(K_M, cfg.H // cfg.H_G, axis=1).reshape(m_end - i_end, -1)
+        tol, _ = hp.score_error_bound(Q64.reshape(l_C, -1), K_rep, cfg.eps)
+        got = ctx.read_pooled_scores(0, m_end - i_end).astype(np.float64)
+        err = np.abs(got - sp.astype(np.float64))
+        assert np.all(err <= tol), f"pooled full-dimension scores off by {err.max():.3e} (bound {tol[np.argmax(err)]:.3e})"
+        assert got.max() == 0.0 and np.all(got <= 0)
+    return sel_gpu
+
+
+@pytest.mark.parametrize("per_head", [False, True])
+@pytest.mark.parametrize("t,l_C", [(3968, 128), (4000, 77), (4100, 1), (2000, 5), (640, 128)])
+def test_select_full_c1(t, l_C, per_head):
+    _select_full_case(syn.get_config("c1"), t, l_C, per_head)
+
+
+@pytest.mark.parametrize("per_head", [False, True])
+def test_select_full_llama_shape(per_head):
+    _select_full_case(syn.get_config("c2"), 8192, 512, per_head)
+    _select_full_case(syn.get_config("c2"), 9000, 1, per_head)
+
+
+def test_recall_of_the_compressed_selection_against_the_full_dimension_one():
+    """Fig. 3's metric on the mixture-with-needles workload: the share of the full-dimension
+    selection (Eq. 3) that the compressed selection (Eq. 6) also picks.  The kernels' recall equals
+    the oracle's (random-init compressors: the number itself is not a quality claim)."""
+    cfg = syn.get_config("c5")
+    p = hp.oracle_params(cfg)
+    _, _, Wq, Wk = hp.oracle_weights(cfg)
+    t, l_C = 32 * 512, 512
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_batch=1)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, B=1)
+    seq.fill_kv(0, n)
+    fill_kc_gpu(ctx, seq, t)
+    Qb = syn.qkv_rows(cfg, "q", t, n)
+    Q = hp.bits_to_torch(Qb)[None].contiguous()
+    ctx.select(Q, seq.Kc, [t], seq.idx, seq.n_sel, sync=True)
+    sel_c = seq.idx[0, : int(seq.n_sel[0])].cpu().numpy().astype(np.int64)
+    ctx.select_full(Q, seq.K, [t], seq.idx, seq.n_sel, sync=True)
+    sel_f = seq.idx[0, : int(seq.n_sel[0])].cpu().numpy().astype(np.int64)
+    Q64, K64 = syn.bf16_bits_to_f64(Qb), hp.torch_to_f64(seq.K[0])
+    i_end, m_end = orc.partition(t, cfg.l_I, cfg.l_L)
+    res = orc.esa_step(Q64, K64, K64, Wq, Wk, p, t, do_attend=False)
+    sel_f_or, _ = orc.select_full(Q64, K64[i_end:m_end], cfg.k, cfg.eps)
+    want = orc.recall(res.sel_abs, sel_f_or + i_end)
+    got = orc.recall(sel_c, sel_f)
+    print(f"recall of the compressed selection: kernels {got:.4f}, oracle {want:.4f}")
+    assert abs(got - want) <= 2.0 / cfg.k
+
+
 # ------------------------------------------------ two-position attention (Section 3.2)
 def _two_position_case(cfg, t, l_C, heads=None, use_qfar=True, use_kfar=True, n_sel=None, seed=0):
     """esa_attend_two_position against the oracle: I and M_k attended with a second encoding of the

@@ -277,6 +277,66 @@ def test_attend_subset_matches_library_with_explicit_mask():
     assert np.allclose(got, sdpa_ref(Q, K, V, vis, 0.37), rtol=1e-10, atol=1e-12)
 
 
+# ------------------------------------------- full-dimension and per-head scores
+def test_full_dimension_score_is_the_dot_product_of_concatenated_heads():
+    """Eq. 3 equals one dot product of the H concatenated heads (keys of a GQA group repeated),
+    as Section 3.1 states; also against explicit loops."""
+    g = rng(31)
+    l_C, l_M, H, H_G, d = 5, 11, 6, 2, 4
+    Q = rand_bf16(g, l_C, H, d)
+    K = rand_bf16(g, l_M, H_G, d)
+    S = orc.scores_full(Q, K)
+    K_rep = np.repeat(K, H // H_G, axis=1)                     # [l_M, H, d]
+    want = (Q.reshape(l_C, H * d) @ K_rep.reshape(l_M, H * d).T).astype(np.float32)
+    assert np.array_equal(S, want)
+    brute = np.zeros((l_C, l_M))
+    for c in range(l_C):
+        for m in range(l_M):
+            for h in range(H):
+                for i in range(d):
+                    brute[c, m] += Q[c, h, i] * K[m, h // (H // H_G), i]
+    assert np.allclose(S, brute, rtol=1e-6, atol=1e-6)
+
+
+def test_per_head_vote_bruteforce_and_reductions():
+    g = rng(32)
+    l_C, l_M, H, H_G, d = 4, 9, 4, 2, 4
+    Q = rand_bf16(g, l_C, H, d)
+    K = rand_bf16(g, l_M, H_G, d)
+    got = orc.aggregate_per_head(Q, K)
+    want = np.full(l_M, -np.inf)
+    for h in range(H):
+        S_h = np.array([[np.float32(Q[c, h] @ K[m, h // 2]) for m in range(l_M)] for c in range(l_C)], np.float32)
+        for m in range(l_M):
+            for c in range(l_C):
+                want[m] = max(want[m], np.float32(S_h[c, m] - S_h[c].max()))
+    assert np.array_equal(got, want.astype(np.float32))
+    assert got.max() == 0.0 and np.all(got <= 0)
+    # with a single head the vote and the summed score coincide
+    Q1, K1 = Q[:, :1], K[:, :1]
+    assert np.array_equal(orc.aggregate_per_head(Q1, K1), orc.aggregate(orc.scores_full(Q1, K1)))
+    sel_u, sp_u = orc.select_full(Q1, K1, 3, 1)
+    sel_i, sp_i = orc.select_full(Q1, K1, 3, 1, per_head=True)
+    assert np.array_equal(sel_u, sel_i) and np.array_equal(sp_u, sp_i)
+
+
+def test_compression_with_an_orthonormal_basis_reproduces_the_full_scores():
+    """When the two compressors are the same orthonormal basis of the whole space (d' = d_H), the
+    compressed score q' . k' (Eq. 6) is the full-dimension score (Eq. 3), so both selections agree
+    and the recall is 1.  Entries are small integers so that every step is exact."""
+    g = rng(33)
+    l_C, l_M, H, d = 3, 40, 2, 4
+    Q = np.round(4 * g.standard_normal((l_C, H, d)))
+    K = np.round(4 * g.standard_normal((l_M, H, d)))
+    P = np.eye(H * d)[g.permutation(H * d)]                    # a permutation: orthonormal, exact in bf16
+    qc, kc = orc.compress(Q.reshape(l_C, -1), P), orc.compress(K.reshape(l_M, -1), P)
+    sel_c, sp_c, _ = orc.select(qc, kc, 7, 1)
+    sel_f, sp_f = orc.select_full(Q, K, 7, 1)
+    assert np.array_equal(sp_c, sp_f) and np.array_equal(sel_c, sel_f)
+    assert orc.recall(sel_c, sel_f) == 1.0
+    assert orc.recall(np.array([1, 2, 3]), np.array([2, 3, 4, 5])) == 0.5
+
+
 def test_attention_by_parts_equals_single_softmax():
     """Algorithm 1: a causal part on [L, C] and a non-causal part on [I, M_k], merged by the
     softmax of their log-normalisers, equal one softmax over the union; so does any other cut."""
