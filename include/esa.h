@@ -182,6 +182,26 @@ esa_status esa_attend_two_position_async(esa_ctx* ctx, int32_t B, const void* Q_
                                          const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel, void* O,
                                          void* stream);
 
+/* Appendix "Model Loading": the K/V cache offloaded to host memory, the compressed keys on
+ * the GPU, and only the attended rows brought onto the GPU at every step (the paper's
+ * single-GPU mode for contexts of 700k+ tokens).  esa_attend with host-resident caches:
+ *   K_host, V_host   [B, max_tokens, H_G, d] in page-locked host memory that the device can
+ *                    address (cudaHostAlloc / cudaHostRegister; pass the device-side pointer,
+ *                    which equals the host pointer under unified addressing).  They already
+ *                    hold C at rows [n_prev[b], n_prev[b] + l_C).
+ *   K_stage, V_stage device [B, stage_rows, H_G, d] scratch owned by the caller, stage_rows >=
+ *                    l_I + top_k + l_L + l_C: the rows of I, M_k, L and C are copied there in
+ *                    list order by one gather kernel (16-byte reads across PCIe), and the
+ *                    attention kernels run on the staged rows.
+ * Everything else is as for esa_attend; the result is bit-identical to esa_attend on
+ * device-resident copies of the same caches.  ESA_ERR_CAPACITY if stage_rows is too small. */
+esa_status esa_attend_host_kv(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_host,
+                              const void* V_host, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
+                              void* K_stage, void* V_stage, int64_t stage_rows, void* O);
+esa_status esa_attend_host_kv_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_host,
+                                    const void* V_host, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
+                                    void* K_stage, void* V_stage, int64_t stage_rows, void* O, void* stream);
+
 /* (No counterpart in the paper: an integration convenience.)
  * esa_attend for small chunks -- l_C * (H / H_G) <= 64 rows, the decode case -- that needs
  * neither a context nor any allocation.  It is for callers that may not allocate device

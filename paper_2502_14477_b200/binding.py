@@ -91,6 +91,11 @@ _PROTOS = {
     "esa_attend_two_position_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                 C.c_void_p]),
+    "esa_attend_host_kv": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "esa_attend_host_kv_async": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                           C.c_void_p]),
     "esa_attend_noalloc": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "esa_read_pooled_scores": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
@@ -332,6 +337,34 @@ class Esa:
                                                         _ptr(O), _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_attend_two_position")
+
+    def attend_host_kv(self, Q_cur, K_host, V_host, n_prev, idx, n_sel, K_stage, V_stage, O, stream=None, sync=False):
+        """``esa_attend_host_kv``: K_host / V_host are pinned host tensors [B, max_tokens, H_G, d]; K_stage / V_stage
+        device scratch [B, stage_rows, H_G, d]."""
+        c = self.cfg
+        B, l_C = Q_cur.shape[0], Q_cur.shape[1]
+        _check(Q_cur, "Q_cur", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        for t, name in ((K_host, "K_host"), (V_host, "V_host")):
+            if t.is_cuda or not t.is_pinned():
+                raise TypeError(f"{name} must be a pinned host tensor")
+            if t.dtype != torch.bfloat16 or not t.is_contiguous() or t.shape != (B, c.max_tokens, c.n_kv_heads, c.head_dim):
+                raise ValueError(f"{name} must be contiguous bf16 [B, max_tokens, H_G, d]")
+        stage_rows = K_stage.shape[1]
+        _check(K_stage, "K_stage", torch.bfloat16, (B, stage_rows, c.n_kv_heads, c.head_dim))
+        _check(V_stage, "V_stage", torch.bfloat16, (B, stage_rows, c.n_kv_heads, c.head_dim))
+        _check(idx, "idx", torch.int32, (B, c.top_k))
+        _check(n_sel, "n_sel", torch.int32, (B,))
+        _check(O, "O", torch.bfloat16, (B, l_C, c.n_q_heads, c.head_dim))
+        npv = self._nprev(n_prev, B)
+        if sync:
+            st = self.lib.esa_attend_host_kv(self._h, B, _ptr(Q_cur), l_C, K_host.data_ptr(), V_host.data_ptr(), npv, _ptr(idx),
+                                             _ptr(n_sel), _ptr(K_stage), _ptr(V_stage), stage_rows, _ptr(O))
+        else:
+            st = self.lib.esa_attend_host_kv_async(self._h, B, _ptr(Q_cur), l_C, K_host.data_ptr(), V_host.data_ptr(), npv,
+                                                   _ptr(idx), _ptr(n_sel), _ptr(K_stage), _ptr(V_stage), stage_rows, _ptr(O),
+                                                   _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_attend_host_kv")
 
     def read_pooled_scores(self, b: int, n: int, stream=None) -> np.ndarray:
         out = np.empty(n, dtype=np.float32)

@@ -443,6 +443,43 @@ esa_status esa_attend(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, c
     return from_cuda(cudaStreamSynchronize(nullptr));
 }
 
+// ------------------------------------------------------- host-resident K/V
+esa_status esa_attend_host_kv_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_host,
+                                    const void* V_host, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
+                                    void* K_stage, void* V_stage, int64_t stage_rows, void* O, void* stream) {
+    esa_status s = check_common(ctx, B);
+    if (s != ESA_OK) return s;
+    if (!Q_cur || !K_host || !V_host || !n_prev || !idx || !n_sel || !K_stage || !V_stage || !O || l_C <= 0)
+        return ESA_ERR_INVALID_ARG;
+    if (l_C > ctx->cfg.max_chunk) return ESA_ERR_CAPACITY;
+    SeqMeta meta;
+    s = build_meta(ctx, B, n_prev, l_C, &meta, nullptr);
+    if (s != ESA_OK) return s;
+    // rows of the attended list per sequence (the selection may hold fewer than top_k: the upper bound sizes the stage)
+    for (int b = 0; b < B; ++b) {
+        const int lM = meta.m_end[b] - meta.i_end[b];
+        const int64_t n_att = (int64_t)meta.i_end[b] + (lM < ctx->cfg.top_k ? lM : ctx->cfg.top_k) + (meta.t[b] - meta.m_end[b]) + l_C;
+        if (n_att > stage_rows) return ESA_ERR_CAPACITY;
+    }
+    if (stage_rows >= (int64_t(1) << 31)) return ESA_ERR_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (launch_gather_kv(ctx, B, l_C, K_host, V_host, meta, idx, n_sel, K_stage, V_stage, stage_rows, st) != cudaSuccess)
+        return ESA_ERR_CUDA;
+    // The staged rows are the attended list itself: the attention kernels run on the same partition with the
+    // identity as the map from list positions to cache rows.
+    return from_cuda(launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, nullptr, (const __nv_bfloat16*)K_stage, nullptr,
+                                   (const __nv_bfloat16*)V_stage, meta, idx, n_sel, (__nv_bfloat16*)O, st, stage_rows, true));
+}
+
+esa_status esa_attend_host_kv(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_host,
+                              const void* V_host, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
+                              void* K_stage, void* V_stage, int64_t stage_rows, void* O) {
+    esa_status s = esa_attend_host_kv_async(ctx, B, Q_cur, l_C, K_host, V_host, n_prev, idx, n_sel, K_stage, V_stage,
+                                            stage_rows, O, nullptr);
+    if (s != ESA_OK) return s;
+    return from_cuda(cudaStreamSynchronize(nullptr));
+}
+
 // --------------------------------------------------------------- diagnostics
 esa_status esa_read_pooled_scores(esa_ctx* ctx, int32_t b, float* dst_host, int64_t n, void* stream) {
     if (!ctx || !dst_host || b < 0 || b >= ctx->cfg.max_batch || n < 0) return ESA_ERR_INVALID_ARG;
@@ -481,7 +518,7 @@ const char* esa_kernel_class_name(int32_t cls) {
         "score_tc_kernel<.,2>", "score_pass_kernel<.,1>+<.,2>", "score_decode_kernel", "score_full_kernel<.,1>+<.,2>",
         "pool_hist_kernel",
         "select_topk_kernel", "select_all_kernel", "attend_tc_kernel", "attend_decode_kernel", "attend_kernel",
-        "attend_merge_kernel"};
+        "attend_merge_kernel", "gather_kv_kernel"};
     return cls >= 0 && cls < KC_COUNT ? names[cls] : "";
 }
 

@@ -38,6 +38,7 @@ struct AttendParams {
     float* part;              // split partials
     int* unit_count;          // arrival counters per (sequence, key/value head) for the in-kernel merge of the decode kernel
     int* status;              // device status word (may be null: the entry point without a context)
+    int staged;               // the caches hold the attended list itself: row j = list entry j
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
@@ -101,7 +102,8 @@ attend_kernel(AttendParams p) {
             bool ok = j < n_att;
             int pos = 0;
             if (ok) {
-                if (j < i_end) pos = j;
+                if (p.staged) pos = j;
+                else if (j < i_end) pos = j;
                 else if (j < n_glob) pos = clamp_selected(__ldg(idx + (j - i_end)), i_end, m_end, bad_idx);
                 else pos = m_end + (j - n_glob);
             }
@@ -431,7 +433,7 @@ attend_decode_kernel(AttendParams p) {
             if (TWO && j < n_glob) far_mask |= 1u << i;
             int q = -1;
             if (it < it_end && j < n_att) {
-                if (j < i_end) q = j;
+                if (p.staged || j < i_end) q = j;
                 else if (j < n_glob) {
                     q = __ldg(idx + (j - i_end));
                     sel_mask |= 1u << i;
@@ -743,13 +745,15 @@ static cudaError_t launch_small(esa_ctx* ctx, AttendParams& p, int B, int l_C, i
 // Qg / Kg: queries and key cache used against I and M_k (Section 3.2); null = Q / K.
 cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
                           const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
-                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st) {
+                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st, int64_t cache_rows,
+                          bool staged) {
     const bool two = (Qg && Qg != Q) || (Kg && Kg != K);
     AttendParams p;
     p.Q = Q; p.K = K; p.Qg = Qg ? Qg : Q; p.Kg = Kg ? Kg : K;
     p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
     p.status = ctx->status;
-    p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
+    p.staged = staged ? 1 : 0;
+    p.max_tokens = cache_rows > 0 ? cache_rows : ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
     p.meta = meta;
@@ -764,7 +768,7 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
         // prefill-sized chunks: tcgen05 kernel (a split key list is merged inside it)
         int nsplit = 1;
         return launch_attend_tc(ctx, B, l_C, Q, two ? p.Qg : nullptr, K, two ? p.Kg : nullptr, V, meta, idx, n_sel, O, n_att_max, st,
-                                &nsplit);
+                                &nsplit, cache_rows, staged);
     }
     return two ? launch_small<true>(ctx, p, B, l_C, n_att_max, st) : launch_small<false>(ctx, p, B, l_C, n_att_max, st);
 }
@@ -875,7 +879,7 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
     AttendParams p;
     p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
     p.Qg = p.Q; p.Kg = p.K;
-    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr;
+    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr; p.staged = 0;
     p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
     p.top_k = cfg->top_k; p.nsplit = 1;
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)D);

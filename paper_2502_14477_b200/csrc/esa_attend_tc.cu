@@ -77,6 +77,7 @@ struct TcAttendParams {
     int Rp;             // rows of a scratch part (R rounded up to even: 16-byte aligned parts)
     int* unit_count;    // arrivals per (sequence, key/value head, row tile); returns to 0 after each launch
     int q_tma;          // Q tiles arrive by TMA (one arrival) instead of cp.async (one per producer thread)
+    int staged;         // the caches hold the attended list itself: row j = list entry j
     float scale_log2;
     SeqMeta meta;
 };
@@ -600,7 +601,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 const int jj = key0 + rsub + it * RSTEP;
                 int q = -1;
                 if (jj >= row_lim) q = -1;
-                else if (jj < i_end) q = jj;
+                else if (p.staged || jj < i_end) q = jj;
                 else if (jj < n_glob) {
                     q = __ldg(idx + (jj - i_end));
                     from_idx |= 1u << it;
@@ -746,13 +747,14 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
 cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
                              const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
                              const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, int n_att_max, cudaStream_t st,
-                             int* nsplit_out) {
+                             int* nsplit_out, int64_t cache_rows, bool staged) {
     const bool two = Qg != nullptr || Kg != nullptr;
     TcAttendParams p;
     p.Q = Q; p.K = K; p.Qg = Qg ? Qg : Q; p.Kg = Kg ? Kg : K;
     p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.status = ctx->status;
     p.unit_count = ctx->att_count;
-    p.max_tokens = ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
+    p.staged = staged ? 1 : 0;
+    p.max_tokens = cache_rows > 0 ? cache_rows : ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
     p.meta = meta;

@@ -46,7 +46,7 @@ struct RowMap {
 enum KernelClass {
     KC_COMPRESS_TC = 0, KC_COMPRESS_GEMV, KC_COMPRESS_MMA, KC_APPEND_KV, KC_SCORE_PASS1, KC_SCORE_PASS2, KC_SCORE_MMA,
     KC_SCORE_DECODE, KC_SCORE_FULL, KC_POOL_HIST, KC_SELECT_TOPK, KC_SELECT_ALL, KC_ATTEND_TC, KC_ATTEND_DECODE, KC_ATTEND_SMALL,
-    KC_ATTEND_MERGE, KC_COUNT
+    KC_ATTEND_MERGE, KC_GATHER_KV, KC_COUNT
 };
 struct ProfRec {
     int cls;
@@ -162,9 +162,17 @@ cudaError_t launch_select_all(esa_ctx* ctx, int B, const SeqMeta& meta, int32_t*
                               int32_t* n_sel_out, cudaStream_t st);
 
 // Qg / Kg: queries and key cache used against I and M_k (two-position attention, Section 3.2); null = Q / K.
+// cache_rows: rows per sequence of the K/V caches handed in (0 = the configuration's max_tokens).
+// staged: the caches hold the attended list itself, row j = list entry j (host-resident K/V, staged by launch_gather_kv).
 cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
                           const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
-                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st);
+                          const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O, cudaStream_t st,
+                          int64_t cache_rows = 0, bool staged = false);
+
+// Host-resident K/V: copies the rows of the attended list, in list order, into device staging caches.
+cudaError_t launch_gather_kv(esa_ctx* ctx, int B, int l_C, const void* K_host, const void* V_host, const SeqMeta& meta,
+                             const int32_t* idx, const int32_t* n_sel, void* K_stage, void* V_stage, int64_t stage_rows,
+                             cudaStream_t st);
 
 // Prefill-sized chunks (l_C * H/H_G > kAttSplitRows) on tcgen05; *nsplit_out reports the number of
 // key-list splits (their partials pass through ctx->att_part and are merged inside the kernel).
@@ -172,7 +180,7 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
 cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, const __nv_bfloat16* Qg,
                              const __nv_bfloat16* K, const __nv_bfloat16* Kg, const __nv_bfloat16* V, const SeqMeta& meta,
                              const int32_t* idx, const int32_t* n_sel, __nv_bfloat16* O,
-                             int n_att_max, cudaStream_t st, int* nsplit_out);
+                             int n_att_max, cudaStream_t st, int* nsplit_out, int64_t cache_rows = 0, bool staged = false);
 
 // TMA descriptor of a row-major bf16 matrix [rows, cols] (cols a multiple of 64), read in boxes of
 // box_rows x 64 columns with the 128-byte swizzle.  False when the driver entry point is missing

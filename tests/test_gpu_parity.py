@@ -534,6 +534,49 @@ def test_two_position_attention_llama_shape_and_group_of_seven():
     _two_position_case(cfg, 10000, 1)
 
 
+# ------------------------------------------------ host-resident K/V (appendix "Model Loading")
+@pytest.mark.parametrize("name,t,l_C,n_sel", [("c1", 3968, 128, None), ("c1", 4100, 1, None), ("c1", 2000, 5, 100),
+                                               ("c1", 300, 128, None), ("c2", 8192, 512, None), ("c2", 9000, 1, None)])
+def test_attention_with_host_resident_kv(name, t, l_C, n_sel):
+    """The K/V cache lives in pinned host memory; the attended rows are staged on the device by the
+    library's gather kernel.  Same bits as esa_attend on device-resident copies, and within the
+    attention tolerance of the oracle."""
+    cfg = syn.get_config(name)
+    p = hp.oracle_params(cfg)
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=1)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, B=1)
+    seq.fill_kv(0, n)
+    K_host = seq.K.cpu().pin_memory()
+    V_host = seq.V.cpu().pin_memory()
+    Qb = syn.qkv_rows(cfg, "q", t, n)
+    Q = hp.bits_to_torch(Qb)[None].contiguous()
+    i_end, m_end = orc.partition(t, cfg.l_I, cfg.l_L)
+    kk = min(cfg.k, m_end - i_end) if n_sel is None else n_sel
+    g = np.random.default_rng(5)
+    sel = np.sort(g.choice(np.arange(i_end, m_end), size=kk, replace=False)) if kk else np.zeros(0, np.int64)
+    seq.idx[0, :kk] = torch.from_numpy(sel.astype(np.int32)).cuda()
+    seq.n_sel[0] = kk
+    stage_rows = cfg.l_I + cfg.k + cfg.l_L + l_C
+    K_stage = torch.zeros(1, stage_rows, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda")
+    V_stage = torch.zeros_like(K_stage)
+    O_host = torch.full_like(Q, float("nan"))
+    ctx.attend_host_kv(Q, K_host, V_host, [t], seq.idx, seq.n_sel, K_stage, V_stage, O_host, sync=True)
+    O_dev = torch.empty_like(Q)
+    ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O_dev, sync=True)
+    assert ctx.last_device_status() == 0
+    assert torch.equal(O_host, O_dev)
+    want = orc.attend(syn.bf16_bits_to_f64(Qb), hp.torch_to_f64(seq.K[0]), hp.torch_to_f64(seq.V[0]), sel, t, p,
+                      heads=[0, cfg.H - 1])
+    hp.check_attention(O_host[0], want, what=f"host K/V {name} t={t} l_C={l_C}", heads=[0, cfg.H - 1])
+    # a stage that cannot hold the list is refused before anything is launched
+    import paper_2502_14477_b200 as esa
+    small = torch.zeros(1, 16, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(esa.EsaError) as e:
+        ctx.attend_host_kv(Q, K_host, V_host, [t], seq.idx, seq.n_sel, small, small.clone(), O_host, sync=True)
+    assert e.value.status == 3
+
+
 # ------------------------------------------------------- device-side safety nets
 @pytest.mark.parametrize("t,l_C", [(3000, 1), (3000, 5), (2944, 128)])
 def test_selected_position_outside_M_is_clamped_and_reported(t, l_C):
