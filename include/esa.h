@@ -230,6 +230,25 @@ esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const void* Q_cu
                               const void* K_cache, const void* V_cache, const int64_t* n_prev,
                               const int32_t* idx, const int32_t* n_sel, void* O, void* stream);
 
+/* Eq. 7: fitting the two compressors.  A trainer holds W_q [d_c, H*d], b_q, W_k [d_c, H_G*d], b_k
+ * and their Adam moments on the device (fp32).  One step takes a batch of n query-key pairs
+ * (Q_batch device bf16 [n, H, d], K_batch device bf16 [n, H_G, d], n <= batch), forms the full-dimension
+ * scores q_c k_m^T of all n x n pairs (Eq. 3), the compressed ones f_q(q_c) . f_k(k_m), the mean
+ * squared difference and its gradients, and applies one Adam update (beta 0.9 / 0.999, eps 1e-8,
+ * no weight decay; the paper names no optimiser, Section 4.1 gives the learning rate 5e-4, batches
+ * of 128 and 10 epochs).  loss_out: device fp32, receives the loss before the update (may be NULL).
+ * Used fields of cfg: n_q_heads, n_kv_heads, head_dim, d_c.  esa_fit_set_weights installs host fp32
+ * initial values (biases may be NULL = 0) and resets the optimiser; esa_fit_get_weights synchronises
+ * the device and copies the current values to host memory (pass them to esa_set_compressors). */
+typedef struct esa_fit esa_fit;
+esa_status esa_fit_create(const esa_config* cfg, int32_t batch, float lr, esa_fit** out);
+esa_status esa_fit_destroy(esa_fit* fit);
+esa_status esa_fit_set_weights(esa_fit* fit, const float* Wq, const float* bq, const float* Wk, const float* bk);
+esa_status esa_fit_get_weights(esa_fit* fit, float* Wq, float* bq, float* Wk, float* bk);
+esa_status esa_fit_step_async(esa_fit* fit, const void* Q_batch, const void* K_batch, int32_t n, float* loss_out,
+                              void* stream);
+int64_t esa_fit_launch_count(const esa_fit* fit);
+
 /* Diagnostic: copies the pooled scores s' (Eq. 8) of the most recent esa_select of
  * sequence b to host memory dst[0..n) as fp32, n <= number of middle tokens of that
  * call.  Synchronises the given stream.  ESA_ERR_STATE if that call did no scoring. */

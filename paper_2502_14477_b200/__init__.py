@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     EsaError,
     EsaConfig,
     Esa,
+    EsaFit,
     load_library,
     library_path,
     STATUS_NAMES,
@@ -15,4 +16,4 @@ from .binding import (  # noqa: F401
 )
 from .build import build_library  # noqa: F401
 
-__all__ = ["EsaError", "EsaConfig", "Esa", "load_library", "library_path", "build_library", "STATUS_NAMES", "attend_noalloc"]
+__all__ = ["EsaError", "EsaConfig", "Esa", "EsaFit", "load_library", "library_path", "build_library", "STATUS_NAMES", "attend_noalloc"]

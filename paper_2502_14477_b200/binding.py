@@ -98,6 +98,12 @@ _PROTOS = {
                                            C.c_void_p]),
     "esa_attend_noalloc": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_fit_create": (C.c_int, [C.POINTER(_CConfig), C.c_int32, C.c_float, C.POINTER(C.c_void_p)]),
+    "esa_fit_destroy": (C.c_int, [C.c_void_p]),
+    "esa_fit_set_weights": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_fit_get_weights": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "esa_fit_step_async": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "esa_fit_launch_count": (C.c_int64, [C.c_void_p]),
     "esa_read_pooled_scores": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]),
     "esa_read_compressed_queries": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "esa_debug_wait_timeout": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p]),
@@ -401,6 +407,61 @@ class Esa:
         st = self.lib.esa_debug_wait_timeout(self._h, int(limit_cycles), _stream_ptr(stream))
         if st != 0:
             raise EsaError(st, "esa_debug_wait_timeout")
+
+
+class EsaFit:
+    """Trainer of the two compressors (Eq. 7): ``esa_fit_*``.  Marshalling only."""
+
+    def __init__(self, cfg: EsaConfig, batch: int, lr: float = 5e-4):
+        self.lib = load_library()
+        self.cfg, self.batch = cfg, batch
+        self._c = cfg.to_c()
+        h = C.c_void_p()
+        st = self.lib.esa_fit_create(C.byref(self._c), batch, lr, C.byref(h))
+        if st != 0:
+            raise EsaError(st, "esa_fit_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self.lib.esa_fit_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launch_count(self) -> int:
+        return int(self.lib.esa_fit_launch_count(self._h))
+
+    def set_weights(self, Wq, bq, Wk, bk):
+        arr = [None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.float32)) for a in (Wq, bq, Wk, bk)]
+        st = self.lib.esa_fit_set_weights(self._h, *[None if a is None else a.ctypes.data_as(C.c_void_p) for a in arr])
+        if st != 0:
+            raise EsaError(st, "esa_fit_set_weights")
+
+    def get_weights(self):
+        c = self.cfg
+        out = (np.empty((c.d_c, c.n_q_heads * c.head_dim), np.float32), np.empty(c.d_c, np.float32),
+               np.empty((c.d_c, c.n_kv_heads * c.head_dim), np.float32), np.empty(c.d_c, np.float32))
+        st = self.lib.esa_fit_get_weights(self._h, *[a.ctypes.data_as(C.c_void_p) for a in out])
+        if st != 0:
+            raise EsaError(st, "esa_fit_get_weights")
+        return out
+
+    def step(self, Q_batch, K_batch, loss_out=None, stream=None):
+        c = self.cfg
+        n = Q_batch.shape[0]
+        _check(Q_batch, "Q_batch", torch.bfloat16, (n, c.n_q_heads, c.head_dim))
+        _check(K_batch, "K_batch", torch.bfloat16, (n, c.n_kv_heads, c.head_dim))
+        if loss_out is not None:
+            _check(loss_out, "loss_out", torch.float32, (1,))
+        st = self.lib.esa_fit_step_async(self._h, _ptr(Q_batch), _ptr(K_batch), n, _ptr(loss_out), _stream_ptr(stream))
+        if st != 0:
+            raise EsaError(st, "esa_fit_step_async")
 
 
 def attend_noalloc(cfg: EsaConfig, Q_cur, K_cache, V_cache, n_prev, idx, n_sel, O, stream=None):

@@ -542,3 +542,68 @@ def test_needles_are_selected_full_size_chunk():
     cfg = syn.get_config("c5")
     hit, tot, n = _needle_recall(cfg, 1, 7)
     assert tot >= 16 and hit == tot and n == cfg.k
+
+
+# ------------------------------------------------------- compressor fitting (Eq. 7)
+def _fit_problem(g, n=6, H=4, H_G=2, d=3, dc=2):
+    from oracle import esa_fit_oracle as fo
+    Q = g.standard_normal((n, H, d))
+    K = g.standard_normal((n, H_G, d))
+    P = {"Wq": 0.3 * g.standard_normal((dc, H * d)), "bq": 0.1 * g.standard_normal(dc),
+         "Wk": 0.3 * g.standard_normal((dc, H_G * d)), "bk": 0.1 * g.standard_normal(dc)}
+    return fo, Q, K, P
+
+
+def test_fit_target_is_the_full_dimension_score():
+    g = rng(41)
+    fo, Q, K, _ = _fit_problem(g)
+    T = fo.fold_heads(Q, K.shape[1]) @ K.reshape(K.shape[0], -1).T
+    assert np.allclose(T, orc.scores_full(Q, K).astype(np.float64), rtol=1e-6, atol=1e-6)
+
+
+def test_fit_gradients_match_finite_differences():
+    g = rng(42)
+    fo, Q, K, P = _fit_problem(g)
+    loss, dWq, dbq, dWk, dbk = fo.loss_and_grads(Q, K, P["Wq"], P["bq"], P["Wk"], P["bk"])
+    grads = {"Wq": dWq, "bq": dbq, "Wk": dWk, "bk": dbk}
+    h = 1e-6
+    for name in grads:
+        flat = P[name].reshape(-1)
+        for i in range(0, flat.size, max(1, flat.size // 5)):
+            old = flat[i]
+            flat[i] = old + h
+            lp = fo.loss_and_grads(Q, K, P["Wq"], P["bq"], P["Wk"], P["bk"])[0]
+            flat[i] = old - h
+            lm = fo.loss_and_grads(Q, K, P["Wq"], P["bq"], P["Wk"], P["bk"])[0]
+            flat[i] = old
+            assert abs((lp - lm) / (2 * h) - grads[name].reshape(-1)[i]) <= 1e-5 * max(1.0, abs(grads[name].reshape(-1)[i])), name
+
+
+def test_first_adam_step_moves_by_lr_against_the_gradient_sign():
+    g = rng(43)
+    fo, Q, K, P = _fit_problem(g)
+    before = {k: v.copy() for k, v in P.items()}
+    grads = dict(zip(("Wq", "bq", "Wk", "bk"), fo.loss_and_grads(Q, K, P["Wq"], P["bq"], P["Wk"], P["bk"])[1:]))
+    st = fo.AdamState(lr=5e-4)
+    fo.fit_step(P, Q, K, st)
+    for name in P:
+        assert np.allclose(P[name] - before[name], -5e-4 * np.sign(grads[name]), rtol=1e-4, atol=1e-9)
+
+
+def test_fit_reaches_near_zero_loss_when_the_data_lie_in_a_small_subspace():
+    """Queries and keys confined to a d'-dimensional subspace (one head, no grouping) admit exact
+    compressors -- the projection on that subspace -- so the loss can be driven towards zero."""
+    from oracle import esa_fit_oracle as fo
+    g = rng(44)
+    D, dc, n = 12, 3, 16
+    basis = np.linalg.qr(g.standard_normal((D, dc)))[0]             # [D, dc] orthonormal columns
+    P = {"Wq": 0.5 * g.standard_normal((dc, D)), "bq": np.zeros(dc), "Wk": 0.5 * g.standard_normal((dc, D)), "bk": np.zeros(dc)}
+    st = fo.AdamState(lr=2e-2)
+    first = last = None
+    for it in range(1500):
+        Q = (g.standard_normal((n, dc)) @ basis.T)[:, None, :]
+        K = (g.standard_normal((n, dc)) @ basis.T)[:, None, :]
+        loss = fo.fit_step(P, Q, K, st)
+        first = loss if first is None else first
+        last = loss
+    assert last < 1e-3 * first
