@@ -527,6 +527,91 @@ def time_prefill_leg(name, steps, peaks):
     return out
 
 
+def time_extensions(peaks):
+    """The steps next to the measured path, each on the c5 shape (512 queries after 65536 cached tokens unless
+    noted), timed with the library's per-kernel CUDA events over a few repetitions: two-position attention
+    (Section 3.2), full-dimension and per-head selection (Eq. 3, Section 4.3), attention with the K/V cache
+    in host memory (appendix "Model Loading") and compressor fitting (Eq. 7)."""
+    import paper_2502_14477_b200 as esa
+    cfg = syn.get_config("c5")
+    t, l_C, reps = 65536, cfg.l_C, 5
+    n = t + l_C
+    ctx = make_ctx(cfg, n, l_C, 1)
+    wq, wk = syn.compressor_weights(cfg)
+    ctx.set_compressors(wq, None, wk, None)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    mk = lambda *shape: torch.randn(*shape, device="cuda", dtype=torch.bfloat16, generator=g)
+    K, V, Kf = mk(1, n, cfg.H_G, cfg.d), mk(1, n, cfg.H_G, cfg.d), mk(1, n, cfg.H_G, cfg.d)
+    Q, Qf = mk(1, l_C, cfg.H, cfg.d), mk(1, l_C, cfg.H, cfg.d)
+    idx = torch.zeros(1, cfg.k, dtype=torch.int32, device="cuda")
+    n_sel = torch.zeros(1, dtype=torch.int32, device="cuda")
+    O = torch.empty_like(Q)
+    i_end, l_M, n_att = partition_sizes(cfg, t, l_C)
+    idx[0] = (torch.sort(torch.randperm(l_M, device="cuda", generator=g)[: cfg.k])[0] + i_end).to(torch.int32)
+    n_sel[0] = cfg.k
+    out = {"shape": f"c5 shape, {l_C} queries after {t} cached tokens, {reps} repetitions each, inputs drawn on the device"}
+
+    def timed(fn, name):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ctx.read_profile()
+        ctx.set_profiling(True)
+        for _ in range(reps):
+            fn()
+        ctx.set_profiling(False)
+        torch.cuda.synchronize()
+        return {k: 1e3 * ms / cnt for k, (cnt, ms) in ctx.read_profile().items()}
+
+    fl_att = attend_flops(cfg, t, l_C)
+    one = timed(lambda: ctx.attend(Q, K, V, [t], idx, n_sel, O), "attend")["attend_tc_kernel"]
+    two = timed(lambda: ctx.attend_two_position(Q, Qf, K, Kf, V, [t], idx, n_sel, O), "attend2")["attend_tc_kernel"]
+    out["two_position_attention"] = {"us_per_launch": two, "one_position_us_per_launch": one,
+                                     "achieved_tflops": fl_att / two * 1e-6, "frac_burst": fl_att / two * 1e-6 / peaks["tflops_burst"]}
+    fl_full = 2.0 * 2.0 * cfg.d_H * l_C * l_M          # two passes over all heads and dimensions
+    for per_head, key in ((False, "select_full_uniform"), (True, "select_full_per_head")):
+        pr = timed(lambda: ctx.select_full(Q, K, [t], idx, n_sel, per_head=per_head), key)
+        us = pr["score_full_kernel<.,1>+<.,2>"]
+        out[key] = {"score_us_per_call": us, "achieved_tflops": fl_full / us * 1e-6, "frac_burst": fl_full / us * 1e-6 / peaks["tflops_burst"],
+                    "pool_hist_us": pr.get("pool_hist_kernel"), "select_topk_us": pr.get("select_topk_kernel"),
+                    "note": "mma.sync kernels (both passes timed together); flops = 2 passes x 2 d_H l_C l_M"}
+    idx[0] = (torch.sort(torch.randperm(l_M, device="cuda", generator=g)[: cfg.k])[0] + i_end).to(torch.int32)
+    n_sel[0] = cfg.k
+    K_host, V_host = K.cpu().pin_memory(), V.cpu().pin_memory()
+    stage_rows = cfg.l_I + cfg.k + cfg.l_L + l_C
+    Ks = torch.empty(1, stage_rows, cfg.H_G, cfg.d, dtype=torch.bfloat16, device="cuda")
+    Vs = torch.empty_like(Ks)
+    pr = timed(lambda: ctx.attend_host_kv(Q, K_host, V_host, [t], idx, n_sel, Ks, Vs, O), "host")
+    gbytes = 2.0 * n_att * cfg.d_G * 2
+    out["host_resident_kv"] = {"gather_us": pr["gather_kv_kernel"], "attend_us": pr["attend_tc_kernel"],
+                               "gathered_bytes": gbytes, "host_to_device_gbs": gbytes / pr["gather_kv_kernel"] * 1e-3,
+                               "note": "rows of I, M_k, L, C read from pinned host memory by the gather kernel (PCIe-bound)"}
+    ctx.close()
+    # Eq. 7: fitting steps at the Llama shape, batches of 128 pairs
+    nb, steps = 128, 60
+    fit = esa.EsaFit(esa.EsaConfig(cfg.H, cfg.H_G, cfg.d, cfg.d_c, cfg.l_I, cfg.l_L, cfg.k, cfg.eps, 1, 1, 16), nb, 5e-4)
+    fit.set_weights(wq, None, wk, None)
+    Qb, Kb = mk(nb, cfg.H, cfg.d), mk(nb, cfg.H_G, cfg.d)
+    for _ in range(5):
+        fit.step(Qb, Kb)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fit.step(Qb, Kb)
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / steps
+    fl = 4.0 * nb * cfg.d_c * (cfg.d_H + cfg.d_G) + 2.0 * nb * nb * (cfg.d_G + 3 * cfg.d_c)
+    out["compressor_fitting"] = {"us_per_step": us, "steps_per_s": 1e6 / us, "achieved_tflops_fp32": fl / us * 1e-6,
+                                 "launches_per_step": fit.launch_count / (steps + 5), "bound": "launch latency / fp32 ALU",
+                                 "note": "batch of 128 pairs, fp32 kernels; the paper's 10 epochs over 50k pairs are 3900 such steps"}
+    fit.close()
+    del K, V, Kf, K_host, V_host
+    torch.cuda.empty_cache()
+    return out
+
+
 def profile_case(args):
     """Small, self-ending cases for ncu captures: every kernel of one ESA step, ``--reps`` times, on
     inputs larger than L2 but well under a few GB.  Inputs are N(0,1) bf16 drawn on the device."""
@@ -696,6 +781,7 @@ def run_esa(args, cfg):
     if not args.no_legs:
         for name in ("c2", "c4"):
             legs["prefill_" + name] = time_prefill_leg(name, 2, peaks)
+        legs["extensions"] = time_extensions(peaks)
 
     if rank != 0:
         if world > 1:

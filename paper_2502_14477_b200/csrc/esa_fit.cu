@@ -28,6 +28,7 @@ struct esa_fit {
     float* m1;                    // Adam first moments
     float* m2;                    // Adam second moments
     float *Qf, *T, *A, *Bm, *dP, *dA, *dBm;
+    float* part;                  // partial sums of split reductions
     float* loss_acc;              // one float
     int64_t launches;
 };
@@ -41,13 +42,16 @@ constexpr int GK = 16;
 __device__ __forceinline__ float ldf(const float* p, int64_t i) { return p[i]; }
 __device__ __forceinline__ float ldf(const __nv_bfloat16* p, int64_t i) { return __bfloat162float(p[i]); }
 
-// C[m, n] = alpha * sum_k A(m, k) B(n, k) + bias[n] - sub[m, n], fp32 accumulation in the order of k.
+// C[m, n] = sum_k A(m, k) B(n, k) + bias[n] - sub[m, n], fp32 accumulation in the order of k.
 // A(m, k) = A[m * sam + k * sak], B(n, k) = B[n * sbn + k * sbk]: any of the four transpose
-// combinations by strides.  64 x 64 output tile per CTA, 4 x 4 outputs per thread.
+// combinations by strides.  64 x 64 output tile per CTA, 4 x 4 outputs per thread.  A long reduction
+// is cut into gridDim.z ranges of kslice columns: CTA z then writes its raw partial sums to
+// C + z * M * N, and fit_reduce_kernel adds the partials in the order of z (so the result does not
+// depend on scheduling) and applies bias and sub.
 template <typename TA, typename TB>
 __global__ void __launch_bounds__(256) fit_gemm_kernel(const TA* __restrict__ A, int64_t sam, int64_t sak, const TB* __restrict__ B,
                                                        int64_t sbn, int64_t sbk, float* __restrict__ C, int M, int N, int K,
-                                                       const float* __restrict__ bias, const float* __restrict__ sub) {
+                                                       int kslice, const float* __restrict__ bias, const float* __restrict__ sub) {
     __shared__ float sA[GK][GT + 1];
     __shared__ float sB[GK][GT + 1];
     const int tid = threadIdx.x;
@@ -58,7 +62,12 @@ __global__ void __launch_bounds__(256) fit_gemm_kernel(const TA* __restrict__ A,
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    for (int k0 = 0; k0 < K; k0 += GK) {
+    const int k_begin = blockIdx.z * kslice;
+    if (gridDim.z > 1) {
+        K = min(K, k_begin + kslice);
+        C += (int64_t)blockIdx.z * M * N;
+    }
+    for (int k0 = k_begin; k0 < K; k0 += GK) {
         for (int e = tid; e < GT * GK; e += 256) {
             // the faster-varying index follows the operand's unit stride
             const int r = sak == 1 ? e / GK : e % GT, kk = sak == 1 ? e % GK : e / GT;
@@ -93,6 +102,18 @@ __global__ void __launch_bounds__(256) fit_gemm_kernel(const TA* __restrict__ A,
                 C[(int64_t)m * N + n] = v;
             }
         }
+}
+
+// C[e] = sum over z (in order) of part[z][e] + bias[e % N] - sub[e]
+__global__ void fit_reduce_kernel(const float* __restrict__ part, int splits, float* __restrict__ C, int M, int N,
+                                  const float* __restrict__ bias, const float* __restrict__ sub) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= M * N) return;
+    float v = 0.f;
+    for (int z = 0; z < splits; ++z) v += part[(int64_t)z * M * N + e];
+    if (bias) v += bias[e % N];
+    if (sub) v -= sub[e];
+    C[e] = v;
 }
 
 // Qf[c, g, i] = sum over the heads h of group g of Q[c, h, i] (fp32)
@@ -151,10 +172,24 @@ __global__ void fit_adam_kernel(float* __restrict__ p, const float* __restrict__
     }
 }
 
+// `part`: scratch for split reductions (kFitMaxSplit * M * N floats), or null to reduce in one CTA per tile
+constexpr int kFitMaxSplit = 32;
 template <typename TA, typename TB>
-void gemm(cudaStream_t st, const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbn, int64_t sbk, float* C, int M, int N, int K,
-          const float* bias = nullptr, const float* sub = nullptr) {
-    fit_gemm_kernel<TA, TB><<<dim3((N + GT - 1) / GT, (M + GT - 1) / GT), 256, 0, st>>>(A, sam, sak, B, sbn, sbk, C, M, N, K, bias, sub);
+int gemm(cudaStream_t st, const TA* A, int64_t sam, int64_t sak, const TB* B, int64_t sbn, int64_t sbk, float* C, int M, int N, int K,
+         const float* bias = nullptr, const float* sub = nullptr, float* part = nullptr) {
+    const dim3 tiles((N + GT - 1) / GT, (M + GT - 1) / GT);
+    int splits = 1;
+    if (part) {
+        while (splits < kFitMaxSplit && (int)(tiles.x * tiles.y) * splits < 128 && K / (splits * 2) >= 4 * GK) splits *= 2;
+    }
+    if (splits == 1) {
+        fit_gemm_kernel<TA, TB><<<tiles, 256, 0, st>>>(A, sam, sak, B, sbn, sbk, C, M, N, K, K, bias, sub);
+        return 1;
+    }
+    const int kslice = ((K + splits - 1) / splits + GK - 1) / GK * GK;
+    fit_gemm_kernel<TA, TB><<<dim3(tiles.x, tiles.y, splits), 256, 0, st>>>(A, sam, sak, B, sbn, sbk, part, M, N, K, kslice, nullptr, nullptr);
+    fit_reduce_kernel<<<(M * N + 255) / 256, 256, 0, st>>>(part, splits, C, M, N, bias, sub);
+    return 2;
 }
 
 }  // namespace
@@ -179,7 +214,8 @@ esa_status esa_fit_create(const esa_config* cfg, int32_t batch, float lr, esa_fi
     f->launches = 0;
     f->n_params = (size_t)f->dc * f->dH + f->dc + (size_t)f->dc * f->dG + f->dc;
     const size_t n = batch, dc = f->dc;
-    const size_t floats = 4 * f->n_params + n * f->dG + 2 * n * n + 4 * n * dc + 64;
+    const size_t part_floats = 32 * (n * n > n * dc ? n * n : n * dc);
+    const size_t floats = 4 * f->n_params + n * f->dG + 2 * n * n + 4 * n * dc + part_floats + 64;
     if (cudaGetDevice(&f->device) != cudaSuccess || cudaMalloc(&f->base, floats * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
         delete f;
@@ -197,6 +233,7 @@ esa_status esa_fit_create(const esa_config* cfg, int32_t batch, float lr, esa_fi
     f->Bm = p; p += n * dc;
     f->dA = p; p += n * dc;
     f->dBm = p; p += n * dc;
+    f->part = p; p += part_floats;
     f->loss_acc = p;
     if (cudaMemset(f->base, 0, floats * sizeof(float)) != cudaSuccess) {
         cudaFree(f->base);
@@ -259,25 +296,26 @@ esa_status esa_fit_step_async(esa_fit* f, const void* Q_batch, const void* K_bat
     const int dc = f->dc, dH = f->dH, dG = f->dG;
     // targets (Eq. 3 for every pair)
     fit_fold_kernel<<<(unsigned)(((int64_t)n * dG + 255) / 256), 256, 0, st>>>(Q, f->Qf, n, f->H, f->HG, f->d);
-    gemm(st, f->Qf, (int64_t)dG, 1, K, (int64_t)dG, 1, f->T, n, n, dG);
+    int launches = 5;                                  // fold, loss, two column sums, Adam
+    launches += gemm(st, f->Qf, (int64_t)dG, 1, K, (int64_t)dG, 1, f->T, n, n, dG, nullptr, nullptr, f->part);
     // forward
-    gemm(st, Q, (int64_t)dH, 1, Wq, (int64_t)dH, 1, f->A, n, dc, dH, bq);
-    gemm(st, K, (int64_t)dG, 1, Wk, (int64_t)dG, 1, f->Bm, n, dc, dG, bk);
-    gemm(st, f->A, (int64_t)dc, 1, f->Bm, (int64_t)dc, 1, f->dP, n, n, dc, nullptr, f->T);      // E = A Bm^T - T (in dP's buffer)
+    launches += gemm(st, Q, (int64_t)dH, 1, Wq, (int64_t)dH, 1, f->A, n, dc, dH, bq, nullptr, f->part);
+    launches += gemm(st, K, (int64_t)dG, 1, Wk, (int64_t)dG, 1, f->Bm, n, dc, dG, bk, nullptr, f->part);
+    launches += gemm(st, f->A, (int64_t)dc, 1, f->Bm, (int64_t)dc, 1, f->dP, n, n, dc, nullptr, f->T, f->part);      // E = A Bm^T - T (in dP's buffer)
     if (cudaMemsetAsync(f->loss_acc, 0, sizeof(float), st) != cudaSuccess) return ESA_ERR_CUDA;
     fit_loss_kernel<<<32, 256, 0, st>>>(f->dP, f->dP, f->loss_acc, n * n);
     // backward
-    gemm(st, f->dP, (int64_t)n, 1, f->Bm, 1, (int64_t)dc, f->dA, n, dc, n);                      // dA[c, j] = sum_m dP[c, m] Bm[m, j]
-    gemm(st, f->dP, 1, (int64_t)n, f->A, 1, (int64_t)dc, f->dBm, n, dc, n);                      // dBm[m, j] = sum_c dP[c, m] A[c, j]
-    gemm(st, f->dA, 1, (int64_t)dc, Q, 1, (int64_t)dH, f->grads + owq, dc, dH, n);               // dWq[j, i] = sum_c dA[c, j] Q[c, i]
-    gemm(st, f->dBm, 1, (int64_t)dc, K, 1, (int64_t)dG, f->grads + owk, dc, dG, n);
+    launches += gemm(st, f->dP, (int64_t)n, 1, f->Bm, 1, (int64_t)dc, f->dA, n, dc, n);                      // dA[c, j] = sum_m dP[c, m] Bm[m, j]
+    launches += gemm(st, f->dP, 1, (int64_t)n, f->A, 1, (int64_t)dc, f->dBm, n, dc, n);                      // dBm[m, j] = sum_c dP[c, m] A[c, j]
+    launches += gemm(st, f->dA, 1, (int64_t)dc, Q, 1, (int64_t)dH, f->grads + owq, dc, dH, n);               // dWq[j, i] = sum_c dA[c, j] Q[c, i]
+    launches += gemm(st, f->dBm, 1, (int64_t)dc, K, 1, (int64_t)dG, f->grads + owk, dc, dG, n);
     fit_colsum_kernel<<<(dc + 127) / 128, 128, 0, st>>>(f->dA, f->grads + obq, n, dc);
     fit_colsum_kernel<<<(dc + 127) / 128, 128, 0, st>>>(f->dBm, f->grads + obk, n, dc);
     // Adam
     f->step += 1;
     const float c1 = 1.f - std::pow(f->beta1, (float)f->step), c2 = 1.f - std::pow(f->beta2, (float)f->step);
     fit_adam_kernel<<<256, 256, 0, st>>>(f->params, f->grads, f->m1, f->m2, f->n_params, f->lr, f->beta1, f->beta2, f->eps, c1, c2);
-    f->launches += 14;
+    f->launches += launches;
     if (loss_out && cudaMemcpyAsync(loss_out, f->loss_acc, sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return ESA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? ESA_OK : ESA_ERR_CUDA;
