@@ -29,7 +29,7 @@ bool config_ok(const esa_config* c) {
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct Layout {
-    size_t wq, wk, bq, bk, qc, rkey, rkey_heads, skey, pkey, ghist0, cidx, slice_cnt, ticket, att, att_count, status, total;
+    size_t wq, wk, bq, bk, qc, rkey, rkey_heads, skey, pkey, ghist0, ghist1, cidx, slice_cnt, ticket, att, att_count, status, total;
     size_t att_elems, att_count_elems, slice_stride;
 };
 
@@ -48,6 +48,7 @@ Layout make_layout(const esa_config* c) {
     L.skey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.pkey = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.ghist0 = take(4 * (size_t)c->max_batch * 2048);
+    L.ghist1 = take(4 * (size_t)c->max_batch * 2048);
     L.cidx = take(4 * (size_t)c->max_batch * c->max_tokens);
     L.slice_stride = ((size_t)c->max_tokens + 4095) / 4096;
     L.slice_cnt = take(4 * (size_t)c->max_batch * L.slice_stride);
@@ -170,6 +171,7 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->skey = reinterpret_cast<uint32_t*>(base + L.skey);
     c->pkey = reinterpret_cast<uint32_t*>(base + L.pkey);
     c->ghist0 = reinterpret_cast<uint32_t*>(base + L.ghist0);
+    c->ghist1 = reinterpret_cast<uint32_t*>(base + L.ghist1);
     c->cidx = reinterpret_cast<int32_t*>(base + L.cidx);
     c->sel_slice_cnt = reinterpret_cast<int*>(base + L.slice_cnt);
     c->sel_ticket = reinterpret_cast<int*>(base + L.ticket);
@@ -182,6 +184,7 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->status = reinterpret_cast<int*>(base + L.status);
     if (cudaMemset(c->status, 0, 256) != cudaSuccess ||
         cudaMemset(c->sel_ticket, 0, 4 * (size_t)cfg->max_batch) != cudaSuccess ||
+        cudaMemset(c->ghist1, 0, 4 * (size_t)cfg->max_batch * 2048) != cudaSuccess ||
         cudaMemset(c->att_count, 0, 4 * L.att_count_elems) != cudaSuccess) {
         cudaFree(base);
         delete c;
@@ -564,6 +567,7 @@ esa_status esa_last_device_status(esa_ctx* ctx, void* stream) {
         // a kernel that gave up may have left arrival counters of the in-kernel merges behind
         if (cudaMemsetAsync(ctx->att_count, 0, sizeof(int) * ctx->att_count_elems, st) != cudaSuccess) return ESA_ERR_CUDA;
         if (cudaMemsetAsync(ctx->sel_ticket, 0, sizeof(int) * ctx->cfg.max_batch, st) != cudaSuccess) return ESA_ERR_CUDA;
+        if (cudaMemsetAsync(ctx->ghist1, 0, sizeof(uint32_t) * ctx->cfg.max_batch * 2048, st) != cudaSuccess) return ESA_ERR_CUDA;
         return (esa_status)h;
     }
     return ESA_OK;

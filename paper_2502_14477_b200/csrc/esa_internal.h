@@ -76,6 +76,7 @@ struct esa_ctx {
                          // afterwards the selection's candidate keys
     uint32_t* pkey;      // [max_batch, max_tokens] pooled scores s' as ordered keys (l_C = 1: of the pooled raw scores, r not yet subtracted)
     uint32_t* ghist0;    // [max_batch, 2048] histograms of pkey's top 11 bits (first radix digit)
+    uint32_t* ghist1;    // [max_batch, 2048] second-digit histograms of the selection kernel; 0 between launches
     int32_t* cidx;       // [max_batch, max_tokens] positions of the selection's candidates
     int* sel_slice_cnt;  // [max_batch, sel_slice_stride] candidates per slice of the selection kernel (sized for 4096-token slices, the kernel uses larger ones)
     int* sel_ticket;     // [max_batch] arrival tickets of the selection kernel; 0 between launches

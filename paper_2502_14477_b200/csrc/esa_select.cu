@@ -15,15 +15,19 @@
 //      b0 that holds the k-th largest key, and copies the keys that can still matter -- those
 //      not below the lower edge of b0 -- with their positions, in index order, to its slice of
 //      a candidate list; then it draws an arrival ticket.
+//      Along the way the CTAs add up, for the whole sequence, the histogram of the next 11 bits
+//      among the keys of bin b0.
 //   2. the CTA that draws the last ticket of a sequence gathers the candidate lists (a few
-//      thousand entries, shared memory), finds the k-th largest key T among them by radix
-//      passes (11 + 11 + 10 bits), and emits every candidate with key > T plus the first
-//      (k - #greater) candidates with key == T in index order: exactly "lowest index wins",
-//      and the output is ascending.
+//      thousand entries, shared memory).  The second digit of the k-th largest key T comes from
+//      that histogram; the few keys that share T's top 22 bits are ranked directly (a histogram
+//      pass over the last 10 bits if they are many: long runs of equal scores).  Then every
+//      candidate with key > T plus the first (k - #greater) candidates with key == T in index
+//      order are emitted: exactly "lowest index wins", and the output is ascending.
 // With one query per sequence (decode) the scoring kernel pooled the raw scores P; Eq. 4's
-// s' = fl(P - r) is a monotone map of P, so phase 1 maps every key through it, keeps the keys
-// not below the image of b0's lower edge (a superset of what can matter, and at least k of
-// them), and phase 2 runs on the mapped keys: exactly the selection on s', ties included.
+// s' = fl(P - r) is a monotone map of P.  T is found among the P keys as above; phase 1 keeps the
+// keys whose image is not below the image of b0's lower edge (a superset of what can matter, and
+// at least k of them), and the final comparison against T's image runs on the mapped keys: exactly
+// the selection on s', ties (distinct P with equal images included) broken by index.
 #include "esa_internal.h"
 
 namespace esa {
@@ -35,10 +39,12 @@ constexpr int SEL_ROWS = SEL_SLICE / 32;
 constexpr int SEL_BINS = 2048;
 constexpr int SEL_STAGE_CAP = 12288;  // candidates the last CTA can stage in shared memory (keys and positions)
 constexpr int SEL_MAX_SLICES_SMEM = 1024;
+constexpr int SEL_LIST_CAP = 256;     // keys sharing the threshold's top 22 bits that are ranked directly (more: a histogram pass)
 
 struct SelectParams {
     const uint32_t* pkey;   // [B, max_tokens] pooled keys (mapped != 0: of the pooled raw scores P)
     const uint32_t* ghist0; // [B, SEL_BINS] histogram of pkey's top 11 bits
+    uint32_t* ghist1;       // [B, SEL_BINS] histogram of the next 11 bits among the keys of bin b0; 0 between launches
     const uint32_t* rkey;   // [B * l_C] (mapped mode reads r of query 0)
     uint32_t* ckey;         // [B, max_tokens] candidate keys, slice s at s * SEL_SLICE
     int32_t* cidx;          // [B, max_tokens] candidate positions (absolute), same layout
@@ -155,6 +161,8 @@ select_topk_kernel(SelectParams p) {
     __shared__ int warp_tot[33];
     __shared__ uint32_t scan_tmp[SEL_THREADS / 32];
     __shared__ uint32_t sh_found[2];
+    __shared__ uint32_t lst[SEL_LIST_CAP];         // last CTA: the keys that share the threshold's top 22 bits
+    __shared__ uint32_t lst_n;
     __shared__ uint32_t warp_cnt[2][SEL_THREADS / 32];
     __shared__ int sh_last;
 
@@ -189,23 +197,36 @@ select_topk_kernel(SelectParams p) {
     const uint32_t krem0 = sh_found[1];            // keys of bin b0 among the k largest
     const uint32_t edge = b0 << 21;                // smallest key of bin b0
     const uint32_t cut = mapped ? f32_to_key(key_to_f32(edge) - r0) : edge;
-    if (mapped) {
-#pragma unroll
-        for (int j = 0; j < SEL_PER; ++j) key[j] = f32_to_key(key_to_f32(key[j]) - r0);
-    }
-    // candidates in index order: row r = j * 16 + warp holds tokens base + 32 r .. + 31
+    // (the candidate lists keep the keys as they came; `final_key` is the key the order is decided on)
+    auto final_key = [&](uint32_t kv) { return mapped ? f32_to_key(key_to_f32(kv) - r0) : kv; };
+    // second radix digit of the keys of bin b0, for the whole sequence: every CTA adds its slice's share
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0u;
+    __syncthreads();
+    bool cand[SEL_PER];
 #pragma unroll
     for (int j = 0; j < SEL_PER; ++j) {
         const int m = base + j * SEL_THREADS + tid;
-        const uint32_t bal = __ballot_sync(0xffffffffu, m < l_M && key[j] >= cut);
+        cand[j] = m < l_M && final_key(key[j]) >= cut;
+        const bool surv = m < l_M && (key[j] >> 21) == b0;
+        const uint32_t active = __ballot_sync(0xffffffffu, surv);
+        if (surv) hist_add(hist, (key[j] >> 10) & (SEL_BINS - 1), active);
+    }
+    // candidates in index order: row r = j * 32 + warp holds tokens base + 32 r .. + 31
+#pragma unroll
+    for (int j = 0; j < SEL_PER; ++j) {
+        const uint32_t bal = __ballot_sync(0xffffffffu, cand[j]);
         if (lane == 0) row_cnt[j * (SEL_THREADS / 32) + warp] = __popc(bal);
     }
     __syncthreads();
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) {
+        const uint32_t c = hist[i];
+        if (c) atomicAdd(p.ghist1 + (int64_t)b * SEL_BINS + i, c);
+    }
     const int n_cand = block_exclusive_scan(row_cnt, SEL_ROWS, warp_tot);
 #pragma unroll
     for (int j = 0; j < SEL_PER; ++j) {
         const int m = base + j * SEL_THREADS + tid;
-        const bool take = m < l_M && key[j] >= cut;
+        const bool take = cand[j];
         const uint32_t bal = __ballot_sync(0xffffffffu, take);
         if (take) {
             const int pos = base + row_cnt[j * (SEL_THREADS / 32) + warp] + __popc(bal & ((1u << lane) - 1u));
@@ -326,37 +347,57 @@ select_topk_kernel(SelectParams p) {
     }
     __syncthreads();
 
-    // ---- k-th largest candidate key: radix passes over the dense list
-    uint32_t prefix = 0, krem = (uint32_t)k;
-    const int shifts[3] = {21, 10, 0};
-    const int nbits[3] = {11, 11, 10};
-    int first_pass = 0;
-    if (!mapped) {
-        // the first digit is known from the global histogram (candidates are the keys of bins >= b0)
-        prefix = b0 << 21;
-        krem = krem0;
-        first_pass = 1;
+    // ---- k-th largest pooled key T: its first digit is b0 (global histogram), its second comes from the
+    // histogram the CTAs of phase 1 added up; the handful of keys that share those 22 bits are ranked directly
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) {
+        hist[i] = __ldcg(p.ghist1 + (int64_t)b * SEL_BINS + i);
+        p.ghist1[(int64_t)b * SEL_BINS + i] = 0u;                     // ready for the next launch
     }
-#pragma unroll 1
-    for (int pass = first_pass; pass < 3; ++pass) {
+    if (tid == 0) lst_n = 0u;
+    __syncthreads();
+    find_bin(hist, SEL_BINS, krem0, scan_tmp, sh_found);
+    const uint32_t top22 = (b0 << 11) | sh_found[0];
+    const uint32_t krem1 = sh_found[1];
+    for (int i = tid; i < C; i += SEL_THREADS) {
+        const uint32_t kv = dk[i];
+        if ((kv >> 10) == top22) {
+            const uint32_t at = atomicAdd(&lst_n, 1u);
+            if (at < SEL_LIST_CAP) lst[at] = kv;
+        }
+    }
+    __syncthreads();
+    const uint32_t n_lst = lst_n;
+    if (n_lst <= SEL_LIST_CAP) {
+        if (tid < (int)n_lst) {
+            const uint32_t kv = lst[tid];
+            uint32_t g = 0, e = 0;
+            for (uint32_t j = 0; j < n_lst; ++j) {
+                const uint32_t o = lst[j];
+                g += o > kv;
+                e += o == kv;
+            }
+            if (g < krem1 && krem1 <= g + e) sh_found[0] = kv;         // (every key equal to T writes the same value)
+        }
+        __syncthreads();
+    } else {
+        // many keys share the 22 bits (long runs of equal scores): one more histogram pass over the last 10 bits
         for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
         __syncthreads();
-        const int sh = shifts[pass];
-        const uint32_t dmask = (1u << nbits[pass]) - 1u;
-        const int psh = pass == 0 ? 32 : shifts[pass - 1];     // bits psh and above are fixed
         for (int i0 = warp * 32; i0 < C; i0 += SEL_THREADS) {
             const int i = i0 + lane;
             const uint32_t kv = i < C ? dk[i] : 0u;
-            const bool take = i < C && (pass == 0 || (kv >> psh) == (prefix >> psh));
+            const bool take = i < C && (kv >> 10) == top22;
             const uint32_t active = __ballot_sync(0xffffffffu, take);
-            if (take) hist_add(hist, (kv >> sh) & dmask, active);
+            if (take) hist_add(hist, kv & 1023u, active);
         }
         __syncthreads();
-        find_bin(hist, 1 << nbits[pass], krem, scan_tmp, sh_found);
-        prefix |= sh_found[0] << sh;
-        krem = sh_found[1];
+        find_bin(hist, 1024, krem1, scan_tmp, sh_found);
+        if (tid == 0) sh_found[0] |= top22 << 10;
+        __syncthreads();
     }
-    const uint32_t T = prefix;
+    // the order is decided on the final keys: Eq. 4's subtraction is monotone, so the k-th largest final key
+    // is the image of the k-th largest pooled key
+    const uint32_t T = final_key(sh_found[0]);
 
     // ---- ordered compaction: each warp owns a contiguous run of 32-candidate rows
     const int rows = (C + 31) / 32;
@@ -365,7 +406,7 @@ select_topk_kernel(SelectParams p) {
     const int w_hi = min(C, (warp + 1) * rows_per_warp * 32);
     uint32_t n_gt = 0, n_eq = 0;
     for (int i = w_lo + lane; i < w_hi; i += 32) {
-        const uint32_t kv = dk[i];
+        const uint32_t kv = final_key(dk[i]);
         n_gt += kv > T;
         n_eq += kv == T;
     }
@@ -397,7 +438,7 @@ select_topk_kernel(SelectParams p) {
     int32_t* out = p.idx_out + (int64_t)b * p.top_k;
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
         const int i = i0 + lane;
-        const uint32_t kv = i < w_hi ? dk[i] : 0u;
+        const uint32_t kv = i < w_hi ? final_key(dk[i]) : 0u;
         const bool gt = i < w_hi && kv > T;
         const bool eq = i < w_hi && kv == T;
         const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
@@ -492,7 +533,7 @@ cudaError_t launch_select(esa_ctx* ctx, int B, bool mapped, const SeqMeta& meta,
         ctx->launches += 1;
     }
     SelectParams p;
-    p.pkey = ctx->pkey; p.ghist0 = ctx->ghist0; p.rkey = ctx->rkey;
+    p.pkey = ctx->pkey; p.ghist0 = ctx->ghist0; p.ghist1 = ctx->ghist1; p.rkey = ctx->rkey;
     p.ckey = ctx->skey; p.cidx = ctx->cidx; p.slice_cnt = ctx->sel_slice_cnt; p.ticket = ctx->sel_ticket;
     p.idx_out = idx_out; p.n_sel_out = n_sel_out;
     p.max_tokens = ctx->cfg.max_tokens; p.slice_stride = ctx->sel_slice_stride; p.top_k = ctx->cfg.top_k;
