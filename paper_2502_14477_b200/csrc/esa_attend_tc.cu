@@ -94,7 +94,8 @@ enum {
                                             // the issuing warp, so one barrier per buffer keeps waits adjacent)
     BAR_PV_DONE = BAR_P_READY + 4,          // per Q tile: 2
     BAR_O_READY = BAR_PV_DONE + 2,          // per Q tile: 2, completes once
-    BAR_COUNT = BAR_O_READY + 2
+    BAR_PAIR = BAR_O_READY + 2,             // PAIR: a column half of the other CTA's partial has landed: 2, complete once
+    BAR_COUNT = BAR_PAIR + 2
 };
 
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
@@ -107,6 +108,23 @@ __device__ __forceinline__ void reg_alloc() {
 template <int N>
 __device__ __forceinline__ void reg_dealloc() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(N));
+}
+// Barrier over all threads of a thread-block cluster, split in two so that warps with nothing to publish
+// can arrive early.  Arrive releases this thread's shared-memory writes, wait acquires the others'.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
+// address of the same shared-memory location in another CTA of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t smem_addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(smem_addr), "r"(cta_rank));
+    return r;
+}
+// Bulk copy from this CTA's shared memory into another CTA's of the cluster; the bytes are counted on the
+// destination CTA's mbarrier.  Addresses and size are multiples of 16.
+__device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes, uint32_t mbar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst_cluster),
+                 "r"(src_cta), "r"(bytes), "r"(mbar_cluster)
+                 : "memory");
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;
@@ -149,11 +167,48 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
     return r;
 }
 
+// The merged rows of one column half (DH columns) leave as bf16 through a per-warp staging buffer: 16-byte
+// stores, whole rows per instruction.  acc: this lane's row; lane rr of the warp owns row wrow0 + rr, whose
+// element offset in O is (own_hi : own_lo).
+template <int DH>
+__device__ __forceinline__ void store_half_rows(const float* acc, float4* stage, int lane, int wrow0, int R, uint32_t own_lo,
+                                                uint32_t own_hi, __nv_bfloat16* O_half) {
+    constexpr int NB = DH / 8;               // uint4 per staged row
+    uint4* st16 = reinterpret_cast<uint4*>(stage);
+#pragma unroll
+    for (int q8 = 0; q8 < NB; ++q8) {
+        uint4 o4;
+        o4.x = pack_bf16(acc[q8 * 8 + 0], acc[q8 * 8 + 1]);
+        o4.y = pack_bf16(acc[q8 * 8 + 2], acc[q8 * 8 + 3]);
+        o4.z = pack_bf16(acc[q8 * 8 + 4], acc[q8 * 8 + 5]);
+        o4.w = pack_bf16(acc[q8 * 8 + 6], acc[q8 * 8 + 7]);
+        st16[lane * NB + (q8 ^ (lane & (NB - 1)))] = o4;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int it = 0; it < NB; ++it) {
+        const int e = it * 32 + lane, rr = e / NB, c = e % NB;
+        const uint32_t lo = __shfl_sync(0xffffffffu, own_lo, rr), hi32 = __shfl_sync(0xffffffffu, own_hi, rr);
+        if (wrow0 + rr < R) {
+            __nv_bfloat16* d2 = O_half + (((int64_t)hi32 << 32) | lo);
+            *reinterpret_cast<uint4*>(d2 + c * 8) = st16[rr * NB + (c ^ (rr & (NB - 1)))];
+        }
+    }
+    __syncwarp();
+}
+
 // TWO (two-position attention): the list entries of I and M_k take their logits from Qg and Kg, the
 // entries of L and C from Q and K.  Both pairs of Q tiles stay in shared memory (three K/V stages instead
 // of four make room), the I u M_k part of the key list is padded to whole tiles so that a tile never
 // mixes the two, and the issuing warp picks the Q tiles by the tile's part.
-template <int D, bool TWO>
+// PAIR: the key list is split in two and the two CTAs of a unit form a thread-block cluster.  The CTA of the
+// second half parks its partial (O, m, l) in its own shared memory (the K/V stages, idle by then); after a
+// cluster barrier (both CTAs have finished their products) it sends the partial into the same place of the
+// other CTA's shared memory with bulk copies, and that CTA, once its mbarrier has counted the bytes, merges
+// it with its own accumulator: no round trip through global memory, no fences, no arrival counter.  (Measured
+// for the 128 KB of a partial: loads from the other CTA's shared memory 9 us, one 16-byte store per lane and
+// row 6 us.)  A second cluster barrier keeps the sender's shared memory alive until the copies have landed.
+template <int D, bool TWO, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap qgmap, TcAttendParams p) {
     constexpr int STAGES = TWO ? 3 : TC_STAGES;
@@ -203,6 +258,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             mbar_init(bar(BAR_PV_DONE + q), 1);
             mbar_init(bar(BAR_O_READY + q), 1);
         }
+        mbar_init(bar(BAR_PAIR), 1);
+        mbar_init(bar(BAR_PAIR + 1), 1);
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512);
@@ -356,6 +413,100 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                     }
                 }
             }
+        } else if (PAIR) {
+            // ---- key list split in two, the two CTAs in one cluster (see the comment above the kernel)
+            constexpr int DH = D / 2;
+            constexpr int NCELL = DH / 4;              // 16-byte cells per parked half row
+            const int rl = qt * 128 + lane_base + lane;                       // row within the CTA
+            uint8_t* park = TWO ? sQg : sK;            // [2 column halves][256][D / 2] fp32, cells XOR-swizzled by the row
+            static_assert((TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES >= TC_ROWS * D * 4, "the parked partial must fit");
+            // both warpgroups have passed their O_READY: no MMA reads the Q tiles or the K/V stages any more
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");
+            // shared memory of the Q tiles: warp w of Q tile q stages its bf16 result in the first half of the 8 KB
+            // at q * 32 KB + w * 8 KB (D = 128); the (m, l) of the other part sit in the unused half of the first one
+            uint8_t* wslot = sQ + qt * Q_TILE_BYTES + (warp_u & 3) * (Q_TILE_BYTES / 4);
+            float2* ml_all = reinterpret_cast<float2*>(sQ + Q_TILE_BYTES / 8);          // [256]
+            static_assert(TC_ROWS * 8 <= 128 * D * 2 / 8, "(m, l) of 256 rows must fit in half a warp slot");
+            constexpr uint32_t HALF_BYTES = TC_ROWS * DH * 4, ML_BYTES = TC_ROWS * 8;
+            if (split == 0 && tid == 0) {
+                mbar_arrive_expect_tx(bar(BAR_PAIR), HALF_BYTES + ML_BYTES);
+                mbar_arrive_expect_tx(bar(BAR_PAIR + 1), HALF_BYTES);
+            }
+            if (split == 1) {
+                float4* prow = reinterpret_cast<float4*>(park) + (size_t)rl * NCELL;        // + h * 256 * NCELL for half h
+                if (n_tiles > 0) {
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c0, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int q4 = 0; q4 < 8; ++q4) {
+                            const int cell = c0 / 4 + q4;    // of the whole row
+                            prow[(cell / NCELL) * (TC_ROWS * NCELL) + ((cell % NCELL) ^ (rl & (NCELL - 1)))] =
+                                make_float4(__uint_as_float(o[4 * q4]), __uint_as_float(o[4 * q4 + 1]),
+                                            __uint_as_float(o[4 * q4 + 2]), __uint_as_float(o[4 * q4 + 3]));
+                        }
+                    }
+                }
+                ml_all[rl] = make_float2(m_run, l_run);      // m = -inf: empty part
+                fence_async_smem();                          // the bulk copies read these writes through the async proxy
+            }
+            cluster_arrive();
+            cluster_wait();
+            if (split == 1 && tid == 0) {
+                // (m, l) and the first column half count on the first barrier, the second half on the second
+                const uint32_t rbar0 = cluster_map(bar(BAR_PAIR), 0), rbar1 = cluster_map(bar(BAR_PAIR + 1), 0);
+                bulk_copy_to_cluster(cluster_map(smem_u32(ml_all), 0), smem_u32(ml_all), ML_BYTES, rbar0);
+                constexpr uint32_t PIECE = HALF_BYTES / 4;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    bulk_copy_to_cluster(cluster_map(smem_u32(park) + i * PIECE, 0), smem_u32(park) + i * PIECE, PIECE, i < 4 ? rbar0 : rbar1);
+            }
+            if (split != 0) cluster_arrive();
+            if (split == 0) {
+                mbar_wait(bar(BAR_PAIR), 0, wc);
+                float4* stage = reinterpret_cast<float4*>(wslot);
+                const int wrow0 = row0 + qt * 128 + lane_base;
+                const int64_t own_off = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;
+                const uint32_t own_lo = (uint32_t)own_off, own_hi = (uint32_t)(own_off >> 32);
+                const float4* prow = reinterpret_cast<const float4*>(park) + (size_t)rl * NCELL;
+                const float2 ml1 = ml_all[rl];
+                // weights of the two parts in the log2 domain (Algorithm 1's merge of (O, m, l)), split order
+                const float m_max = fmaxf(m_run, ml1.x);
+                const float w0 = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_max);
+                const float w1 = (ml1.x == -INFINITY) ? 0.f : fast_exp2(ml1.x - m_max);
+                const float inv = 1.f / (w0 * l_run + w1 * ml1.y);
+                const float a0 = w0 * inv, a1 = w1 * inv;
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    float acc[DH];
+#pragma unroll
+                    for (int cc = 0; cc < DH; cc += 16) {
+                        uint32_t o[16];
+                        tmem_ld16(tO + h * DH + cc, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[cc + i] = (a0 != 0.f) ? a0 * __uint_as_float(o[i]) : 0.f;
+                    }
+                    if (h == 1) {
+                        mbar_wait(bar(BAR_PAIR + 1), 0, wc);
+                        cluster_arrive();                    // everything has landed: the sender may go
+                    }
+                    if (a1 != 0.f) {                         // an empty part may hold anything
+#pragma unroll
+                        for (int c = 0; c < DH / 4; ++c) {
+                            const float4 val = prow[h * (TC_ROWS * NCELL) + (c ^ (rl & (NCELL - 1)))];
+                            acc[4 * c] = fmaf(a1, val.x, acc[4 * c]);
+                            acc[4 * c + 1] = fmaf(a1, val.y, acc[4 * c + 1]);
+                            acc[4 * c + 2] = fmaf(a1, val.z, acc[4 * c + 2]);
+                            acc[4 * c + 3] = fmaf(a1, val.w, acc[4 * c + 3]);
+                        }
+                    }
+                    store_half_rows<DH>(acc, stage, lane, wrow0, R, own_lo, own_hi, p.O + h * DH);
+                }
+            }
+            cluster_wait();
         } else {
             // ---- split key list.  Every CTA leaves its partial (O, m, l) in the scratch; the CTA that
             // finishes a (sequence, head, row tile) unit last combines the others' partials with its own,
@@ -515,32 +666,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                         __syncwarp();
                         if (i + 2 < n_pairs) issue(i + 2);
                     }
-                    // bf16 rows of this half leave through the staging buffer: 16-byte stores, whole rows per instruction
-                    {
-                        constexpr int NB = DH / 8;               // uint4 per staged row
-                        uint4* st16 = reinterpret_cast<uint4*>(stage);
-#pragma unroll
-                        for (int q8 = 0; q8 < NB; ++q8) {
-                            uint4 o4;
-                            o4.x = pack_bf16(acc[q8 * 8 + 0], acc[q8 * 8 + 1]);
-                            o4.y = pack_bf16(acc[q8 * 8 + 2], acc[q8 * 8 + 3]);
-                            o4.z = pack_bf16(acc[q8 * 8 + 4], acc[q8 * 8 + 5]);
-                            o4.w = pack_bf16(acc[q8 * 8 + 6], acc[q8 * 8 + 7]);
-                            st16[lane * NB + (q8 ^ (lane & (NB - 1)))] = o4;
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int it = 0; it < NB; ++it) {
-                            const int e = it * 32 + lane, rr = e / NB, c = e % NB;
-                            // lane rr of this warp owns row wrow0 + rr and knows where it goes
-                            const uint32_t lo = __shfl_sync(0xffffffffu, own_lo, rr), hi32 = __shfl_sync(0xffffffffu, own_hi, rr);
-                            if (wrow0 + rr < R) {
-                                __nv_bfloat16* d2 = p.O + (((int64_t)hi32 << 32) | lo) + h * DH;
-                                *reinterpret_cast<uint4*>(d2 + c * 8) = st16[rr * NB + (c ^ (rr & (NB - 1)))];
-                            }
-                        }
-                        __syncwarp();
-                    }
+                    store_half_rows<D / 2>(acc, stage, lane, wrow0, R, own_lo, own_hi, p.O + h * DH);
                 }
             }
         }
@@ -691,6 +817,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         }
     }
 
+    if (PAIR && warp_u >= TC_SOFTMAX_WARPS) {
+        // the cluster barriers count every thread: the warps with nothing to publish pass both
+        cluster_arrive();
+        cluster_wait();
+        cluster_arrive();
+        cluster_wait();
+    }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 512);
@@ -698,24 +831,51 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
 
 }  // namespace
 
+template <int D, bool TWO, bool PAIR>
+static cudaError_t launch_tc_kernel(esa_ctx* ctx, const CUtensorMap& qmap, const CUtensorMap& qgmap, const TcAttendParams& p,
+                                    dim3 grid, cudaStream_t st, bool probe_only) {
+    constexpr int smem = (TWO ? 4 : 2) * 128 * D * 2 + 2 * (TWO ? 3 : TC_STAGES) * TC_BN * D * 2 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D, TWO, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    // the in-kernel register split assumes the launch allocation it was sized for
+    static int regs_checked = 0;
+    if (!regs_checked) {
+        cudaFuncAttributes fa;
+        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D, TWO, PAIR>);
+        if (e != cudaSuccess) return e;
+        if (fa.numRegs != TC_REGS_LAUNCH) return cudaErrorInvalidConfiguration;
+        regs_checked = 1;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 2;
+    cfg.attrs = attr;
+    cfg.numAttrs = PAIR ? 2 : 1;
+    if (probe_only) {
+        // can the device place a pair of these CTAs at all?
+        int n_clusters = 0;
+        e = cudaOccupancyMaxActiveClusters(&n_clusters, attend_tc_kernel<D, TWO, PAIR>, &cfg);
+        if (e != cudaSuccess) return e;
+        return n_clusters > 0 ? cudaSuccess : cudaErrorNotSupported;
+    }
+    return cudaLaunchKernelEx(&cfg, attend_tc_kernel<D, TWO, PAIR>, qmap, qgmap, p);
+}
+
 template <int D, bool TWO>
 static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_max, cudaStream_t st, int* nsplit_out) {
     const int R = p.l_C * p.G;
     const int row_tiles = (R + TC_ROWS - 1) / TC_ROWS;
     p.Rp = (R + 1) & ~1;
     if ((size_t)B * p.HG * row_tiles > ctx->att_count_elems) return cudaErrorNotSupported;
-    constexpr int smem = (TWO ? 4 : 2) * 128 * D * 2 + 2 * (TWO ? 3 : TC_STAGES) * TC_BN * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    // the in-kernel register split assumes the launch allocation it was sized for
-    static int regs_checked = 0;
-    if (!regs_checked) {
-        cudaFuncAttributes fa;
-        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D, TWO>);
-        if (e != cudaSuccess) return e;
-        if (fa.numRegs != TC_REGS_LAUNCH) return cudaErrorInvalidConfiguration;
-        regs_checked = 1;
-    }
     // Split the key list when that fills the machine better: cost model = waves x tiles per CTA
     // (+1 tile-equivalent of fixed work per CTA), one CTA per SM.
     const int ctas = row_tiles * p.HG * B;
@@ -736,8 +896,13 @@ static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_m
     if (p.q_tma && TWO) p.q_tma = make_tensor_map_q(&qgmap, p.Qg, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
     if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
     if (!p.q_tma || !TWO) memset(&qgmap, 0, sizeof(qgmap));
+    const dim3 grid(row_tiles, p.HG, B * best);
+    // a two-way split runs as CTA pairs that merge through distributed shared memory, where the device can place pairs
+    static int pair_ok = -1;                                 // per instantiation; probed once
+    if (best == 2 && pair_ok < 0) pair_ok = launch_tc_kernel<D, TWO, true>(ctx, qmap, qgmap, p, grid, st, true) == cudaSuccess ? 1 : 0;
     ProfScope prof(ctx, KC_ATTEND_TC, st);
-    e = launch_pdl(attend_tc_kernel<D, TWO>, dim3(row_tiles, p.HG, B * best), dim3(TC_THREADS), smem, st, qmap, qgmap, p);
+    cudaError_t e = (best == 2 && pair_ok == 1) ? launch_tc_kernel<D, TWO, true>(ctx, qmap, qgmap, p, grid, st, false)
+                                                : launch_tc_kernel<D, TWO, false>(ctx, qmap, qgmap, p, grid, st, false);
     ctx->launches += 1;
     return e;
 }
