@@ -335,14 +335,17 @@ static cudaError_t launch_score_t(esa_ctx* ctx, int B, int l_C, const __nv_bfloa
             e = cudaMemsetAsync(ctx->ghist0, 0, sizeof(uint32_t) * (size_t)B * SD_BINS, st);
             if (e != cudaSuccess) return e;
         }
-        // Long chunks: every CTA pays a serial start (clear) and tail (pooling, flush) that its loads do
-        // not cover.  Measured with 8 x 129k tokens: 256 / 512 / 1024 / 2048 tokens per CTA give
-        // 87 / 83 / 78 / 76 us for the whole selection.  Short sequences get shorter chunks so that
-        // there are still a few CTAs per SM.
-        int64_t chunk = ((int64_t)B * max_lM * 2 + 7 * ctx->num_sms - 1) / (7 * ctx->num_sms);
-        chunk = (chunk + SD_THREADS - 1) / SD_THREADS * SD_THREADS;
-        if (chunk > SD_TOKENS) chunk = SD_TOKENS;
-        if (chunk < SD_THREADS) chunk = SD_THREADS;
+        // Tokens per CTA.  All CTAs are resident at once and the kernel ends with the SM that got the most work,
+        // so the choice minimises (CTAs on the fullest SM) x (tokens per CTA + the CTA's serial start and tail:
+        // clear, pooling, flush, worth about 256 tokens of loads).  Measured with 8 x 129k tokens: 2048 tokens
+        // per CTA (504 CTAs, four on some SMs and three on others) 55 us, 1792 (576 CTAs, four nearly everywhere)
+        // 52 us, 1536 (672 CTAs, five on some SMs) 71 us.
+        int64_t chunk = SD_THREADS, best_cost = -1;
+        for (int64_t c = SD_THREADS; c <= SD_TOKENS; c += SD_THREADS) {
+            const int64_t n_ctas = (int64_t)B * ((max_lM + c - 1) / c);
+            const int64_t cost = ((n_ctas + ctx->num_sms - 1) / ctx->num_sms) * (c + SD_THREADS);
+            if (best_cost < 0 || cost <= best_cost) { best_cost = cost; chunk = c; }
+        }
         p.chunk = (int)chunk;
         int gx = (max_lM + p.chunk - 1) / p.chunk;
         if (gx < 1) gx = 1;

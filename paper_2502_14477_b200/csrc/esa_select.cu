@@ -234,11 +234,10 @@ select_topk_kernel(SelectParams p) {
             ci[pos] = i_end + m;
         }
     }
-    __threadfence();
+    if (tid == 0) p.slice_cnt[(int64_t)b * p.slice_stride + slice] = n_cand;
+    __threadfence();                                   // every thread's writes (candidates, histogram, count) before the ticket
     __syncthreads();
     if (tid == 0) {
-        p.slice_cnt[(int64_t)b * p.slice_stride + slice] = n_cand;
-        __threadfence();
         const int t = atomicAdd(p.ticket + b, 1);
         sh_last = t == n_slices - 1;
         if (sh_last) p.ticket[b] = 0;              // ready for the next launch
@@ -247,7 +246,21 @@ select_topk_kernel(SelectParams p) {
     if (!sh_last) return;
     __threadfence();
 
-    // ---- phase 2 (one CTA per sequence): offsets of the slices' candidate lists
+    // ---- phase 2 (one CTA per sequence).  The second digit of the k-th largest pooled key T comes from the
+    // histogram the CTAs of phase 1 added up (its first digit is b0); it is read first, so that the keys that
+    // share those 22 bits can be picked out while the candidates pass through the registers on their way to
+    // shared memory.  (The first 32 slice counts are requested at the same time.)
+    const int cnt_first = (warp == 0 && lane < n_slices) ? __ldcg(p.slice_cnt + (int64_t)b * p.slice_stride + lane) : 0;
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) {
+        hist[i] = __ldcg(p.ghist1 + (int64_t)b * SEL_BINS + i);
+        p.ghist1[(int64_t)b * SEL_BINS + i] = 0u;                     // ready for the next launch
+    }
+    if (tid == 0) lst_n = 0u;
+    __syncthreads();
+    find_bin(hist, SEL_BINS, krem0, scan_tmp, sh_found);
+    const uint32_t top22 = (b0 << 11) | sh_found[0];
+    const uint32_t krem1 = sh_found[1];
+    // offsets of the slices' candidate lists:
     // slice counts -> exclusive offsets, SEL_THREADS slices per round (shared memory holds the first
     // SEL_MAX_SLICES_SMEM offsets; longer sequences re-read the counts)
     int* soff = reinterpret_cast<int*>(sel_dyn);   // [n_slices + 1] when it fits, ahead of the staged candidates
@@ -257,7 +270,7 @@ select_topk_kernel(SelectParams p) {
         int run = 0;
         for (int s0 = 0; s0 < n_slices; s0 += 32) {
             const int s = s0 + lane;
-            const int c = s < n_slices ? __ldcg(p.slice_cnt + (int64_t)b * p.slice_stride + s) : 0;
+            const int c = s0 == 0 ? cnt_first : (s < n_slices ? __ldcg(p.slice_cnt + (int64_t)b * p.slice_stride + s) : 0);
             int incl = c;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -311,6 +324,10 @@ select_topk_kernel(SelectParams p) {
                 if (i < C) {
                     skeys[i] = kk[u];
                     sidx[i] = ii[u];
+                    if ((kk[u] >> 10) == top22) {
+                        const uint32_t at = atomicAdd(&lst_n, 1u);
+                        if (at < SEL_LIST_CAP) lst[at] = kk[u];
+                    }
                 }
             }
         }
@@ -347,25 +364,17 @@ select_topk_kernel(SelectParams p) {
     }
     __syncthreads();
 
-    // ---- k-th largest pooled key T: its first digit is b0 (global histogram), its second comes from the
-    // histogram the CTAs of phase 1 added up; the handful of keys that share those 22 bits are ranked directly
-    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) {
-        hist[i] = __ldcg(p.ghist1 + (int64_t)b * SEL_BINS + i);
-        p.ghist1[(int64_t)b * SEL_BINS + i] = 0u;                     // ready for the next launch
-    }
-    if (tid == 0) lst_n = 0u;
-    __syncthreads();
-    find_bin(hist, SEL_BINS, krem0, scan_tmp, sh_found);
-    const uint32_t top22 = (b0 << 11) | sh_found[0];
-    const uint32_t krem1 = sh_found[1];
-    for (int i = tid; i < C; i += SEL_THREADS) {
-        const uint32_t kv = dk[i];
-        if ((kv >> 10) == top22) {
-            const uint32_t at = atomicAdd(&lst_n, 1u);
-            if (at < SEL_LIST_CAP) lst[at] = kv;
+    // ---- k-th largest pooled key T: the handful of keys that share its top 22 bits are ranked directly
+    if (!staged) {
+        for (int i = tid; i < C; i += SEL_THREADS) {
+            const uint32_t kv = dk[i];
+            if ((kv >> 10) == top22) {
+                const uint32_t at = atomicAdd(&lst_n, 1u);
+                if (at < SEL_LIST_CAP) lst[at] = kv;
+            }
         }
+        __syncthreads();
     }
-    __syncthreads();
     const uint32_t n_lst = lst_n;
     if (n_lst <= SEL_LIST_CAP) {
         if (tid < (int)n_lst) {
