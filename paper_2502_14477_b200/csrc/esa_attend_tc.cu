@@ -94,8 +94,8 @@ enum {
                                             // the issuing warp, so one barrier per buffer keeps waits adjacent)
     BAR_PV_DONE = BAR_P_READY + 4,          // per Q tile: 2
     BAR_O_READY = BAR_PV_DONE + 2,          // per Q tile: 2, completes once
-    BAR_PAIR = BAR_O_READY + 2,             // PAIR: a column half of the other CTA's partial has landed: 2, complete once
-    BAR_COUNT = BAR_PAIR + 2
+    BAR_PAIR = BAR_O_READY + 2,             // PAIR: the partner's half of the partial result has landed; completes once
+    BAR_COUNT = BAR_PAIR + 1
 };
 
 __device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
@@ -201,13 +201,15 @@ __device__ __forceinline__ void store_half_rows(const float* acc, float4* stage,
 // entries of L and C from Q and K.  Both pairs of Q tiles stay in shared memory (three K/V stages instead
 // of four make room), the I u M_k part of the key list is padded to whole tiles so that a tile never
 // mixes the two, and the issuing warp picks the Q tiles by the tile's part.
-// PAIR: the key list is split in two and the two CTAs of a unit form a thread-block cluster.  The CTA of the
-// second half parks its partial (O, m, l) in its own shared memory (the K/V stages, idle by then); after a
-// cluster barrier (both CTAs have finished their products) it sends the partial into the same place of the
-// other CTA's shared memory with bulk copies, and that CTA, once its mbarrier has counted the bytes, merges
-// it with its own accumulator: no round trip through global memory, no fences, no arrival counter.  (Measured
-// for the 128 KB of a partial: loads from the other CTA's shared memory 9 us, one 16-byte store per lane and
-// row 6 us.)  A second cluster barrier keeps the sender's shared memory alive until the copies have landed.
+// PAIR: the key list is split in two and the two CTAs of a unit form a thread-block cluster.  CTA r finishes
+// column half r of the unit's rows.  Each parks the other column half of its partial (O, m, l) in its own shared
+// memory (the K/V stages, idle by then); after a cluster barrier (both CTAs have finished their products) each
+// sends that half into the partner's shared memory with bulk copies counted on the partner's mbarrier, and once
+// its own mbarrier has counted the incoming bytes it merges the received half with its accumulator in tensor
+// memory and writes the bf16 rows: no round trip through global memory, no fences, no arrival counter.
+// (Measured for the 128 KB of a partial: loads from the other CTA's shared memory 9 us, one 16-byte store per
+// lane and row 6 us, bulk copies 3.5 us.)  A second cluster barrier keeps each sender's shared memory alive until
+// its copies have landed.
 template <int D, bool TWO, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap qgmap, TcAttendParams p) {
@@ -259,7 +261,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             mbar_init(bar(BAR_O_READY + q), 1);
         }
         mbar_init(bar(BAR_PAIR), 1);
-        mbar_init(bar(BAR_PAIR + 1), 1);
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512);
@@ -414,97 +415,118 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 }
             }
         } else if (PAIR) {
-            // ---- key list split in two, the two CTAs in one cluster (see the comment above the kernel)
+            // ---- key list split in two, the two CTAs in one cluster (see the comment above the kernel).
+            // CTA r finishes column half r of all 256 rows: it sends the other half of its partial and receives
+            // the partner's half r.
             constexpr int DH = D / 2;
-            constexpr int NCELL = DH / 4;              // 16-byte cells per parked half row
+            constexpr int NCELL = DH / 4;              // 16-byte cells per half row
+            constexpr uint32_t HALF_BYTES = TC_ROWS * DH * 4, ML_BYTES = TC_ROWS * 8;
             const int rl = qt * 128 + lane_base + lane;                       // row within the CTA
-            uint8_t* park = TWO ? sQg : sK;            // [2 column halves][256][D / 2] fp32, cells XOR-swizzled by the row
-            static_assert((TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES >= TC_ROWS * D * 4, "the parked partial must fit");
+            // K/V stages (TWO: from the second pair of Q tiles on): [0, HALF_BYTES) the half this CTA sends,
+            // [HALF_BYTES, 2 HALF_BYTES) the half it receives; rows of DH fp32, cells XOR-swizzled by the row
+            uint8_t* park = TWO ? sQg : sK;
+            static_assert((TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES >= 2 * HALF_BYTES, "both halves must fit");
             // both warpgroups have passed their O_READY: no MMA reads the Q tiles or the K/V stages any more
             asm volatile("bar.sync 1, 256;\n" ::: "memory");
             // shared memory of the Q tiles: warp w of Q tile q stages its bf16 result in the first half of the 8 KB
-            // at q * 32 KB + w * 8 KB (D = 128); the (m, l) of the other part sit in the unused half of the first one
+            // at q * 32 KB + w * 8 KB (D = 128); the unused half of the first slot holds this CTA's (m, l), that of the
+            // second slot the partner's
             uint8_t* wslot = sQ + qt * Q_TILE_BYTES + (warp_u & 3) * (Q_TILE_BYTES / 4);
-            float2* ml_all = reinterpret_cast<float2*>(sQ + Q_TILE_BYTES / 8);          // [256]
+            float2* ml_mine = reinterpret_cast<float2*>(sQ + Q_TILE_BYTES / 8);                         // [256]
+            float2* ml_other = reinterpret_cast<float2*>(sQ + Q_TILE_BYTES / 4 + Q_TILE_BYTES / 8);     // [256]
             static_assert(TC_ROWS * 8 <= 128 * D * 2 / 8, "(m, l) of 256 rows must fit in half a warp slot");
-            constexpr uint32_t HALF_BYTES = TC_ROWS * DH * 4, ML_BYTES = TC_ROWS * 8;
-            if (split == 0 && tid == 0) {
-                mbar_arrive_expect_tx(bar(BAR_PAIR), HALF_BYTES + ML_BYTES);
-                mbar_arrive_expect_tx(bar(BAR_PAIR + 1), HALF_BYTES);
-            }
-            if (split == 1) {
-                float4* prow = reinterpret_cast<float4*>(park) + (size_t)rl * NCELL;        // + h * 256 * NCELL for half h
+            const int h_mine = split, h_send = split ^ 1;
+            if (tid == 0) mbar_arrive_expect_tx(bar(BAR_PAIR), HALF_BYTES + ML_BYTES);
+            {
+                float4* prow = reinterpret_cast<float4*>(park) + (size_t)rl * NCELL;
                 if (n_tiles > 0) {
 #pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) {
+                    for (int c0 = 0; c0 < DH; c0 += 32) {
                         uint32_t o[32];
-                        tmem_ld32(tO + c0, o);
+                        tmem_ld32(tO + h_send * DH + c0, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {
-                            const int cell = c0 / 4 + q4;    // of the whole row
-                            prow[(cell / NCELL) * (TC_ROWS * NCELL) + ((cell % NCELL) ^ (rl & (NCELL - 1)))] =
+                        for (int q4 = 0; q4 < 8; ++q4)
+                            prow[(c0 / 4 + q4) ^ (rl & (NCELL - 1))] =
                                 make_float4(__uint_as_float(o[4 * q4]), __uint_as_float(o[4 * q4 + 1]),
                                             __uint_as_float(o[4 * q4 + 2]), __uint_as_float(o[4 * q4 + 3]));
-                        }
                     }
                 }
-                ml_all[rl] = make_float2(m_run, l_run);      // m = -inf: empty part
+                ml_mine[rl] = make_float2(m_run, l_run);     // m = -inf: empty part
                 fence_async_smem();                          // the bulk copies read these writes through the async proxy
             }
             cluster_arrive();
             cluster_wait();
-            if (split == 1 && tid == 0) {
-                // (m, l) and the first column half count on the first barrier, the second half on the second
-                const uint32_t rbar0 = cluster_map(bar(BAR_PAIR), 0), rbar1 = cluster_map(bar(BAR_PAIR + 1), 0);
-                bulk_copy_to_cluster(cluster_map(smem_u32(ml_all), 0), smem_u32(ml_all), ML_BYTES, rbar0);
+            if (tid == 0) {
+                const uint32_t other = split ^ 1;
+                const uint32_t rbar = cluster_map(bar(BAR_PAIR), other);
+                bulk_copy_to_cluster(cluster_map(smem_u32(ml_other), other), smem_u32(ml_mine), ML_BYTES, rbar);
                 constexpr uint32_t PIECE = HALF_BYTES / 4;
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    bulk_copy_to_cluster(cluster_map(smem_u32(park) + i * PIECE, 0), smem_u32(park) + i * PIECE, PIECE, i < 4 ? rbar0 : rbar1);
+                for (int i = 0; i < 4; ++i)
+                    bulk_copy_to_cluster(cluster_map(smem_u32(park) + HALF_BYTES + i * PIECE, other), smem_u32(park) + i * PIECE, PIECE, rbar);
             }
-            if (split != 0) cluster_arrive();
-            if (split == 0) {
-                mbar_wait(bar(BAR_PAIR), 0, wc);
+            mbar_wait(bar(BAR_PAIR), 0, wc);
+            cluster_arrive();                                // the partner's copies have landed here: it may go once it has them too
+            {
                 float4* stage = reinterpret_cast<float4*>(wslot);
                 const int wrow0 = row0 + qt * 128 + lane_base;
                 const int64_t own_off = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;
                 const uint32_t own_lo = (uint32_t)own_off, own_hi = (uint32_t)(own_off >> 32);
-                const float4* prow = reinterpret_cast<const float4*>(park) + (size_t)rl * NCELL;
-                const float2 ml1 = ml_all[rl];
-                // weights of the two parts in the log2 domain (Algorithm 1's merge of (O, m, l)), split order
-                const float m_max = fmaxf(m_run, ml1.x);
-                const float w0 = (m_run == -INFINITY) ? 0.f : fast_exp2(m_run - m_max);
-                const float w1 = (ml1.x == -INFINITY) ? 0.f : fast_exp2(ml1.x - m_max);
-                const float inv = 1.f / (w0 * l_run + w1 * ml1.y);
+                const float4* prow = reinterpret_cast<const float4*>(park + HALF_BYTES) + (size_t)rl * NCELL;
+                const float2 mlo = ml_other[rl];
+                // weights of the two parts in the log2 domain (Algorithm 1's merge of (O, m, l)); part 0 first in every sum
+                const float m0 = split == 0 ? m_run : mlo.x, l0 = split == 0 ? l_run : mlo.y;
+                const float m1 = split == 0 ? mlo.x : m_run, l1 = split == 0 ? mlo.y : l_run;
+                const float m_max = fmaxf(m0, m1);
+                const float w0 = (m0 == -INFINITY) ? 0.f : fast_exp2(m0 - m_max);
+                const float w1 = (m1 == -INFINITY) ? 0.f : fast_exp2(m1 - m_max);
+                const float inv = 1.f / (w0 * l0 + w1 * l1);
                 const float a0 = w0 * inv, a1 = w1 * inv;
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    float acc[DH];
+                const float a_own = split == 0 ? a0 : a1, a_oth = split == 0 ? a1 : a0;
+                float acc[DH];
+                if (split == 0) {
+                    // acc = a0 * own, then += a1 * other
 #pragma unroll
                     for (int cc = 0; cc < DH; cc += 16) {
                         uint32_t o[16];
-                        tmem_ld16(tO + h * DH + cc, o);
+                        tmem_ld16(tO + h_mine * DH + cc, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) acc[cc + i] = (a0 != 0.f) ? a0 * __uint_as_float(o[i]) : 0.f;
+                        for (int i = 0; i < 16; ++i) acc[cc + i] = (a_own != 0.f) ? a_own * __uint_as_float(o[i]) : 0.f;
                     }
-                    if (h == 1) {
-                        mbar_wait(bar(BAR_PAIR + 1), 0, wc);
-                        cluster_arrive();                    // everything has landed: the sender may go
-                    }
-                    if (a1 != 0.f) {                         // an empty part may hold anything
+                    if (a_oth != 0.f) {                      // an empty part may hold anything
 #pragma unroll
-                        for (int c = 0; c < DH / 4; ++c) {
-                            const float4 val = prow[h * (TC_ROWS * NCELL) + (c ^ (rl & (NCELL - 1)))];
-                            acc[4 * c] = fmaf(a1, val.x, acc[4 * c]);
-                            acc[4 * c + 1] = fmaf(a1, val.y, acc[4 * c + 1]);
-                            acc[4 * c + 2] = fmaf(a1, val.z, acc[4 * c + 2]);
-                            acc[4 * c + 3] = fmaf(a1, val.w, acc[4 * c + 3]);
+                        for (int c = 0; c < NCELL; ++c) {
+                            const float4 val = prow[c ^ (rl & (NCELL - 1))];
+                            acc[4 * c] = fmaf(a_oth, val.x, acc[4 * c]);
+                            acc[4 * c + 1] = fmaf(a_oth, val.y, acc[4 * c + 1]);
+                            acc[4 * c + 2] = fmaf(a_oth, val.z, acc[4 * c + 2]);
+                            acc[4 * c + 3] = fmaf(a_oth, val.w, acc[4 * c + 3]);
                         }
                     }
-                    store_half_rows<DH>(acc, stage, lane, wrow0, R, own_lo, own_hi, p.O + h * DH);
+                } else {
+                    // the same sums in the same order: acc = a0 * other, then += a1 * own
+#pragma unroll
+                    for (int c = 0; c < NCELL; ++c) {
+                        const float4 val = prow[c ^ (rl & (NCELL - 1))];
+                        acc[4 * c] = (a_oth != 0.f) ? a_oth * val.x : 0.f;
+                        acc[4 * c + 1] = (a_oth != 0.f) ? a_oth * val.y : 0.f;
+                        acc[4 * c + 2] = (a_oth != 0.f) ? a_oth * val.z : 0.f;
+                        acc[4 * c + 3] = (a_oth != 0.f) ? a_oth * val.w : 0.f;
+                    }
+#pragma unroll
+                    for (int cc = 0; cc < DH; cc += 16) {
+                        uint32_t o[16];
+                        tmem_ld16(tO + h_mine * DH + cc, o);
+                        tmem_wait_ld();
+                        if (a_own != 0.f) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) acc[cc + i] = fmaf(a_own, __uint_as_float(o[i]), acc[cc + i]);
+                        }
+                    }
                 }
+                store_half_rows<DH>(acc, stage, lane, wrow0, R, own_lo, own_hi, p.O + h_mine * DH);
             }
             cluster_wait();
         } else {
