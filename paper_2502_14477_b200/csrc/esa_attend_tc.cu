@@ -21,9 +21,10 @@
 //     the warp-uniform descriptors, lane 0 executes the tcgen05 instructions): a single
 //     diverged thread was starved of issue slots by the arithmetic-heavy softmax warps that
 //     share its scheduler (measured 100-600 cycles per tcgen05.mma instead of 64).
-//   * A quarter of the exponentials is evaluated on the FMA pipe (Cody-Waite split + cubic):
-//     measured pipe rates are 8 cycles per warp for ex2 on the special-function unit against
-//     about 10 FMA/ALU-pipe cycles per polynomial element, so the two pipes balance near 1:3.
+//   * Every exponential is one ex2.approx on the special-function unit.  (Evaluating a share of them on the
+//     FMA pipe -- Cody-Waite split + cubic -- was measured at 1/16, 1/8, 1/4 and 1/2 of the scores: the loop is
+//     bound by the number of instructions the softmax warps issue, not by that unit, and every share was slower
+//     than none.)
 //   * The running maximum is only raised when it grows by more than 2^8: until then the
 //     exponentials are taken against the stale maximum (bounded by 256), which makes
 //     rescaling O in tensor memory rare; (O, m, l) stay consistent, so the final division,
@@ -57,7 +58,6 @@ constexpr int TC_REGS_OTHER = 88;
 static_assert(kAttPrefillSplits == 4, "the in-kernel merge selects among four weights");
 static_assert(8 * TC_REGS_SOFTMAX + 8 * TC_REGS_OTHER <= 16 * TC_REGS_LAUNCH,
               "register split exceeds the CTA's launch allocation: setmaxnreg.inc would never return");
-constexpr int TC_POLY_PAIRS_OF_4 = 1; // of every 4 column pairs, this many take 2^x on the FMA pipe
 constexpr float kRescaleThreshold = 8.0f;    // log2 domain
 
 struct TcAttendParams {
@@ -148,25 +148,6 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
         : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
     return d;
 }
-// 2^x for a pair, x <= ~10, on the FMA pipe: x = n + f with n = round(x), f in [-0.5, 0.5];
-// 2^f by a degree-3 minimax polynomial (relative error 7.5e-5, far below the bf16 rounding
-// of P), n added into the exponent field.  x is clamped at -126 (result ~ 1e-38).
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    const float kMagic = 12582912.0f;                       // 1.5 * 2^23: low mantissa bits hold round(x)
-    x.x = fmaxf(x.x, -126.0f);
-    x.y = fmaxf(x.y, -126.0f);
-    const float2 t = fadd2(x, make_float2(kMagic, kMagic));
-    const float2 n = fadd2(t, make_float2(-kMagic, -kMagic));
-    const float2 f = ffma2(n, make_float2(-1.f, -1.f), x);
-    float2 q = ffma2(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.242611125f, 0.242611125f));
-    q = ffma2(q, f, make_float2(0.693260968f, 0.693260968f));
-    q = ffma2(q, f, make_float2(0.999928057f, 0.999928057f));
-    float2 r;
-    r.x = __uint_as_float(__float_as_uint(q.x) + (__float_as_uint(t.x) << 23));
-    r.y = __uint_as_float(__float_as_uint(q.y) + (__float_as_uint(t.y) << 23));
-    return r;
-}
-
 // The merged rows of one column half (DH columns) leave as bf16 through a per-warp staging buffer: 16-byte
 // stores, whole rows per instruction.  acc: this lane's row; lane rr of the warp owns row wrow0 + rr, whose
 // element offset in O is (own_hi : own_lo).
@@ -366,12 +347,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             for (int i = 0; i < TC_BN / 2; ++i) {
                 const float2 x = ffma2(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2v, nm);
                 float2 e;
-                if ((i & 3) < TC_POLY_PAIRS_OF_4) {
-                    e = exp2_poly2(x);
-                } else {
-                    e.x = fast_exp2(x.x);
-                    e.y = fast_exp2(x.y);
-                }
+                e.x = fast_exp2(x.x);
+                e.y = fast_exp2(x.y);
                 sum4[i & 3] = fadd2(sum4[i & 3], e);
                 pk[i] = pack_bf16(e.x, e.y);
             }
