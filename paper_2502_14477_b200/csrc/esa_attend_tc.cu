@@ -25,10 +25,11 @@
 //     FMA pipe -- Cody-Waite split + cubic -- was measured at 1/16, 1/8, 1/4 and 1/2 of the scores: the loop is
 //     bound by the number of instructions the softmax warps issue, not by that unit, and every share was slower
 //     than none.)
-//   * The running maximum is only raised when it grows by more than 2^8: until then the
-//     exponentials are taken against the stale maximum (bounded by 256), which makes
-//     rescaling O in tensor memory rare; (O, m, l) stay consistent, so the final division,
-//     or the split merge, needs no correction.
+//   * The running maximum m is set on a row's first tile and after that only raised when a tile's sum of
+//     2^(score - m) reaches 2^64: the exponentials are taken against m as it stands, with no search for the
+//     tile's maximum first (one instruction per two scores less in a loop bound by issued instructions) and
+//     hardly ever a rescaling of O in tensor memory; (O, m, l) stay consistent whatever m is, so the final
+//     division, or the split merge, needs no correction, and fp32 (sums, O) and bf16 (P) carry the range.
 //   * A long key list can be split across CTAs (blockIdx.z); partial (O, m, l) go to the
 //     context's scratch through coalesced stores, and the CTA that finishes a unit last merges
 //     them with its own accumulator (an arrival counter per unit decides; nobody waits).
@@ -58,7 +59,7 @@ constexpr int TC_REGS_OTHER = 88;
 static_assert(kAttPrefillSplits == 4, "the in-kernel merge selects among four weights");
 static_assert(8 * TC_REGS_SOFTMAX + 8 * TC_REGS_OTHER <= 16 * TC_REGS_LAUNCH,
               "register split exceeds the CTA's launch allocation: setmaxnreg.inc would never return");
-constexpr float kRescaleThreshold = 8.0f;    // log2 domain
+constexpr float kSumLimit = 1.8446744e19f;   // 2^64: a tile whose sum of 2^(score - m) reaches this has its maximum looked up
 
 struct TcAttendParams {
     const __nv_bfloat16* Q;
@@ -306,18 +307,47 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 for (int i = 0; i < TC_BN; ++i)
                     if (key0 + i >= lim_t) v[i] = 0xff800000u;   // -inf
             }
-            float mxc[8];
+            // P = 2^(S * scale - m) as packed bf16 (it will overwrite the first half of the S buffer); returns the sum
+            // of the tile.  A row without a visible key so far has m = -inf: its P must be 0, not 2^(+inf).
+            uint32_t pk[TC_BN / 2];
+            auto exps = [&](float m) {
+                const float neg_m = (m == -INFINITY) ? 0.f : -m;
+                const float2 sl2v = make_float2(sl2, sl2), nm = make_float2(neg_m, neg_m);
+                float2 sum4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-            for (int c = 0; c < 8; ++c) mxc[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+                for (int i = 0; i < TC_BN / 2; ++i) {
+                    const float2 x = ffma2(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2v, nm);
+                    float2 e;
+                    e.x = fast_exp2(x.x);
+                    e.y = fast_exp2(x.y);
+                    sum4[i & 3] = fadd2(sum4[i & 3], e);
+                    pk[i] = pack_bf16(e.x, e.y);
+                }
+                const float2 a = fadd2(sum4[0], sum4[1]), c = fadd2(sum4[2], sum4[3]);
+                return (a.x + a.y) + (c.x + c.y);
+            };
+            // The exponentials are taken against the running maximum as it stands, without looking for the tile's
+            // own maximum first: (O, m, l) stay consistent whatever m is, and fp32 and bf16 carry the range.  Only when
+            // the tile's sum shows that some score lies far above m (or no key has been seen yet) is the maximum
+            // raised, O rescaled and the tile redone.  The decision is taken per warp: tensor-memory accesses are
+            // warp-wide.
+            float tile_sum = 0.f;
+            bool redo = m_run == -INFINITY;
+            if (!__any_sync(0xffffffffu, redo)) {
+                tile_sum = exps(m_run);
+                redo = !(tile_sum < kSumLimit);              // also true for inf and NaN
+            }
+            if (__any_sync(0xffffffffu, redo)) {
+                float mxc[8];
 #pragma unroll
-            for (int i = 16; i < TC_BN; i += 16)
+                for (int c = 0; c < 8; ++c) mxc[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    mxc[c] = fmax3(mxc[c], __uint_as_float(v[i + 2 * c]), __uint_as_float(v[i + 2 * c + 1]));
-            const float mx = fmaxf(fmax3(mxc[0], mxc[1], mxc[2]), fmax3(fmax3(mxc[3], mxc[4], mxc[5]), mxc[6], mxc[7]));
-            const float m_new = fmaxf(m_run, mx * sl2);
-            const bool grow = m_new > m_run + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, grow)) {
+                for (int i = 16; i < TC_BN; i += 16)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        mxc[c] = fmax3(mxc[c], __uint_as_float(v[i + 2 * c]), __uint_as_float(v[i + 2 * c + 1]));
+                const float mx = fmaxf(fmax3(mxc[0], mxc[1], mxc[2]), fmax3(fmax3(mxc[3], mxc[4], mxc[5]), mxc[6], mxc[7]));
+                const float m_new = fmaxf(m_run, mx * sl2);
                 // 0 on a row's first visible tile; a row that has seen no key yet keeps (m, l) = (-inf, 0)
                 const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
                 l_run *= alpha;
@@ -336,27 +366,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                         tmem_st32(tO + c0, o);
                     }
                 }
-            }
-            // P = 2^(S * scale - m) as packed bf16 over the first half of the S buffer.
-            // A row without a visible key so far has m = -inf: its P must be 0, not 2^(+inf).
-            const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-            const float2 sl2v = make_float2(sl2, sl2), nm = make_float2(neg_m, neg_m);
-            float2 sum4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-            uint32_t pk[TC_BN / 2];
-#pragma unroll
-            for (int i = 0; i < TC_BN / 2; ++i) {
-                const float2 x = ffma2(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2v, nm);
-                float2 e;
-                e.x = fast_exp2(x.x);
-                e.y = fast_exp2(x.y);
-                sum4[i & 3] = fadd2(sum4[i & 3], e);
-                pk[i] = pack_bf16(e.x, e.y);
+                tile_sum = exps(m_run);
             }
             tmem_st32(tS + u * 64, pk);
-            {
-                const float2 a = fadd2(sum4[0], sum4[1]), c = fadd2(sum4[2], sum4[3]);
-                l_run += (a.x + a.y) + (c.x + c.y);
-            }
+            l_run += tile_sum;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BAR_P_READY + qt * 2 + u));
