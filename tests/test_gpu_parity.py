@@ -611,6 +611,52 @@ def test_selected_position_outside_M_is_clamped_and_reported(t, l_C):
     hp.check_attention(O[0], res_O, what="after a clamped index")
 
 
+@pytest.mark.parametrize("name,t,l_C,gain", [("c2", 8192, 512, 12.0), ("c2", 8192, 512, 40.0), ("c1", 3968, 128, 12.0),
+                                              ("c2", 9000, 1, 12.0)])
+def test_attention_with_logits_that_grow_along_the_key_list(name, t, l_C, gain):
+    """Keys scaled up along the positions, so that the largest logit of a row lies tens to hundreds of
+    powers of two above the one its running maximum was set on.  The prefill kernel takes its exponentials
+    against the standing maximum and looks for a tile's own maximum only when the tile's sum overflows its
+    limit: this drives that path (and the rescaling of the accumulator behind it); the other kernels run the
+    same rows through their ordinary online softmax.  Compared with the oracle like every other attention."""
+    cfg = syn.get_config(name)
+    p = hp.oracle_params(cfg)
+    n = t + l_C
+    ctx = hp.make_esa(cfg, max_tokens=n, max_chunk=l_C, max_batch=1)
+    seq = hp.DeviceSeq(cfg, max_tokens=n, B=1)
+    seq.fill_kv(0, n)
+    # K rows grow linearly with the position, to `gain` times their size at the end of the cache (bf16 again)
+    ramp = (1.0 + (gain - 1.0) * torch.arange(n, device="cuda", dtype=torch.float32) / n).view(1, n, 1, 1)
+    seq.K.copy_((seq.K.float() * ramp).to(torch.bfloat16))
+    Qb = syn.qkv_rows(cfg, "q", t, n)
+    Q = hp.bits_to_torch(Qb)[None].contiguous()
+    i_end, m_end = orc.partition(t, cfg.l_I, cfg.l_L)
+    kk = min(cfg.k, m_end - i_end)
+    sel = np.sort(np.random.default_rng(11).choice(np.arange(i_end, m_end), size=kk, replace=False))
+    seq.idx[0, :kk] = torch.from_numpy(sel.astype(np.int32)).cuda()
+    seq.n_sel[0] = kk
+    O = torch.full_like(Q, float("nan"))
+    ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O, sync=True)
+    assert ctx.last_device_status() == 0
+    heads = [0, cfg.H - 1]
+    K64 = hp.torch_to_f64(seq.K[0])
+    want = orc.attend(syn.bf16_bits_to_f64(Qb), K64, hp.torch_to_f64(seq.V[0]), sel, t, p, heads=heads)
+    # the steep case is only worth its name if the logits of a row really span more than the kernel's limit of 2^64
+    q_last = syn.bf16_bits_to_f64(Qb).reshape(l_C, cfg.H, cfg.d)[-1, 0]
+    lg = (K64.reshape(n, cfg.H_G, cfg.d)[:, 0] @ q_last) / np.sqrt(cfg.d) * 1.4426950408889634
+    if gain >= 40.0:
+        assert lg.max() - lg[: cfg.l_I].max() > 64.0, float(lg.max() - lg[: cfg.l_I].max())
+    # With logits this steep a row's weight sits on one or two keys, and the bf16 rounding of that weight (up to
+    # 2^-9 relative, against a sum kept in fp32) goes straight into the output, times the value: the largest
+    # error is bounded relative to the largest value (0.5 %), the mean error by the usual tolerance.
+    got = hp.torch_to_f64(O[0])[:, heads]
+    err = np.abs(got - want[:, heads])
+    vmax = float(np.abs(hp.torch_to_f64(seq.V[0])).max())
+    print(f"growing logits {name} t={t} l_C={l_C} x{gain}: max-abs {err.max():.3e} mean-abs {err.mean():.3e} max|V| {vmax:.2f}")
+    assert np.isfinite(got).all()
+    assert err.max() <= 5e-3 * vmax and err.mean() <= hp.ATT_MEAN_ABS, (float(err.max()), float(err.mean()), vmax)
+
+
 def test_bounded_wait_gives_up_and_the_context_stays_usable():
     """The give-up path of the device-side waits: a wait on a barrier that nothing completes runs
     out after its cycle limit, the kernel returns, the status word says ESA_ERR_TIMEOUT, reading
