@@ -718,12 +718,26 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             }
             cp_async_arrive_noinc(bar(BAR_Q_FULL));
         }
-        const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
-        const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
-        const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + chunk * 8;
+        // K/V tiles: four threads share a row (one instruction of the four covers 64 contiguous bytes of it: whole
+        // sectors), so a thread works out the cache position of two rows per tile, not of eight, and copies CH / 4
+        // chunks of each; the loop is bound by the instructions the CTA's warps issue, these included.
+        constexpr int TPR = 4;                             // threads per row
+        constexpr int RPP = TC_PRODUCERS / TPR;            // rows per pass: 32
+        constexpr int NPASS = TC_BN / RPP;                 // 2
+        constexpr int CPT = CH / TPR;                      // chunks per thread and row: 4 (D = 128) or 2
+        const int q4 = ptid % TPR, rfirst = ptid / TPR;
+        const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
+        const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
+        const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
-        const uint32_t blk_off = (chunk >> 3) * KV_BLK_BYTES;
+        // chunk c = 4 i + q4 of row r goes to block (c >> 3), byte r * 128 + (((c & 7) ^ (r & 7)) << 4) of the tile
+        uint32_t row_off[NPASS];
+#pragma unroll
+        for (int it = 0; it < NPASS; ++it) {
+            const int r = rfirst + it * RPP;
+            row_off[it] = (uint32_t)(r * 128) | (uint32_t)((r & 7) << 4);      // XOR with (c & 7) << 4 gives the swizzled chunk
+        }
         int bad_idx = 0;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % STAGES;
@@ -732,11 +746,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             const bool far = tile_begin + j < far_tiles;
             const int row_lim = far ? far_end : n_att;      // list positions of this tile end here
             const __nv_bfloat16* Ksrc = far ? Kgb : Kb;
-            int pos[TC_BN / RSTEP];
+            int pos[NPASS];
             uint32_t from_idx = 0;                      // rows whose position was read from the selection
 #pragma unroll
-            for (int it = 0; it < TC_BN / RSTEP; ++it) {
-                const int jj = key0 + rsub + it * RSTEP;
+            for (int it = 0; it < NPASS; ++it) {
+                const int jj = key0 + rfirst + it * RPP;
                 int q = -1;
                 if (jj >= row_lim) q = -1;
                 else if (p.staged || jj < i_end) q = jj;
@@ -750,21 +764,31 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             // (the range check of the selected positions comes after the wait: the index loads above stay in
             // flight across it instead of being consumed at once)
 #pragma unroll
-            for (int it = 0; it < TC_BN / RSTEP; ++it)
+            for (int it = 0; it < NPASS; ++it)
                 if ((from_idx >> it) & 1u) pos[it] = clamp_selected(pos[it], i_end, m_end, bad_idx);
 #pragma unroll
-            for (int it = 0; it < TC_BN / RSTEP; ++it) {
-                const int r = rsub + it * RSTEP;
-                uint8_t* dst = sK + s * KV_TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
-                cp_async16(dst, Ksrc + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
+            for (int it = 0; it < NPASS; ++it) {
+                const __nv_bfloat16* src = Ksrc + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
+                const int nbytes = pos[it] < 0 ? 0 : 16;
+                uint8_t* tile = sK + s * KV_TILE_BYTES;
+#pragma unroll
+                for (int i = 0; i < CPT; ++i) {
+                    const int c = i * TPR;                  // + q4: the chunk; (c + q4) & 7 = ((i & 1) * 4 + q4), (c + q4) >> 3 = i >> 1
+                    cp_async16(tile + (i >> 1) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)((((i & 1) * 4 + q4)) << 4)), src + c * 8, nbytes);
+                }
             }
             cp_async_arrive_noinc(bar(BAR_K_FULL + s));
             mbar_wait(bar(BAR_V_EMPTY + s), ph, wc);
 #pragma unroll
-            for (int it = 0; it < TC_BN / RSTEP; ++it) {
-                const int r = rsub + it * RSTEP;
-                uint8_t* dst = sV + s * KV_TILE_BYTES + blk_off + r * 128 + ((cin ^ (r & 7)) << 4);
-                cp_async16(dst, Vb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride, pos[it] < 0 ? 0 : 16);
+            for (int it = 0; it < NPASS; ++it) {
+                const __nv_bfloat16* src = Vb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
+                const int nbytes = pos[it] < 0 ? 0 : 16;
+                uint8_t* tile = sV + s * KV_TILE_BYTES;
+#pragma unroll
+                for (int i = 0; i < CPT; ++i) {
+                    const int c = i * TPR;
+                    cp_async16(tile + (i >> 1) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)((((i & 1) * 4 + q4)) << 4)), src + c * 8, nbytes);
+                }
             }
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
         }
