@@ -731,7 +731,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
-        // chunk c = 4 i + q4 of row r goes to block (c >> 3), byte r * 128 + (((c & 7) ^ (r & 7)) << 4) of the tile
+        // chunk c = TPR i + q4 of row r goes to block (c >> 3), byte r * 128 + (((c & 7) ^ (r & 7)) << 4) of the tile
         uint32_t row_off[NPASS];
 #pragma unroll
         for (int it = 0; it < NPASS; ++it) {
@@ -773,8 +773,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 uint8_t* tile = sK + s * KV_TILE_BYTES;
 #pragma unroll
                 for (int i = 0; i < CPT; ++i) {
-                    const int c = i * TPR;                  // + q4: the chunk; (c + q4) & 7 = ((i & 1) * 4 + q4), (c + q4) >> 3 = i >> 1
-                    cp_async16(tile + (i >> 1) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)((((i & 1) * 4 + q4)) << 4)), src + c * 8, nbytes);
+                    const int c = i * TPR;                  // + q4: the chunk; TPR divides 8, so (c + q4) >> 3 = c >> 3 and (c + q4) & 7 = (c & 7) + q4
+                    cp_async16(tile + (c >> 3) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)(((c & 7) + q4) << 4)), src + c * 8, nbytes);
                 }
             }
             cp_async_arrive_noinc(bar(BAR_K_FULL + s));
@@ -787,7 +787,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
 #pragma unroll
                 for (int i = 0; i < CPT; ++i) {
                     const int c = i * TPR;
-                    cp_async16(tile + (i >> 1) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)((((i & 1) * 4 + q4)) << 4)), src + c * 8, nbytes);
+                    cp_async16(tile + (c >> 3) * KV_BLK_BYTES + (row_off[it] ^ (uint32_t)(((c & 7) + q4) << 4)), src + c * 8, nbytes);
                 }
             }
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
