@@ -4,35 +4,40 @@
 // I u M_k u L u C, C causal), organised for tcgen05:
 //
 //   * A CTA owns 256 rows (row = query c * G + head-in-group g) of one key/value head: two
-//     128-row Q tiles that share every 64-key K/V tile brought into shared memory.
-//   * Scores S = Q K^T and outputs O += P V accumulate in tensor memory.  Per Q tile: two
-//     64-column S buffers (tile j uses buffer j & 1) and D columns of O, 512 columns in all.
-//     P (bf16) overwrites the first half of its own S buffer and is read by the second MMA
-//     straight from tensor memory.
-//   * Because S is double-buffered, Q K^T of tile j + 2 is issued as soon as P V of tile j
-//     has been issued: the softmax of a Q tile never waits for a product it has just asked
-//     for, and the tensor core works through (Q K^T ahead, P V behind) while both softmax
-//     warpgroups compute.  The kernel is bound by the softmax arithmetic, not by a
-//     softmax -> MMA -> softmax chain.
+//     128-row Q tiles that share every 128-key K/V tile brought into shared memory.
+//   * Scores S = Q K^T and outputs O += P V accumulate in tensor memory.  Per Q tile: 128 columns
+//     of S (one 128-key tile, written by products of N = 128: an instruction of N = 64 occupies the
+//     tensor pipe as long as one of N = 128, measured, and with 64-key tiles that pipe bounded the loop)
+//     and D columns of O, 512 columns in all.  The softmax handles a tile as two 64-key halves: P (bf16)
+//     of a half overwrites the first 32 columns of that half and is read by the second MMA straight from
+//     tensor memory, so P V of the first half runs while the exponentials of the second are being taken.
+//   * Per Q tile the chain is S ready -> softmax (two halves) -> P V, then Q K^T of the next tile into
+//     the same columns (the tensor core executes one thread's products in issue order).  One warp issues
+//     for both Q tiles in a fixed alternating order, which keeps them half a period apart: the tensor
+//     core works for one while the other is in its softmax.
 //   * Warp roles: warps 0-3 / 4-7 run the online softmax of Q tile 0 / 1 (one thread per
-//     row holding its 64 scores in registers, so row maxima and sums need no shuffles),
+//     row holding the 64 scores of a half in registers, so row sums need no shuffles),
 //     warps 8-11 gather K/V rows with index-driven 16-byte cp.async into 128-byte-swizzled
-//     tiles, warps 12 and 13 issue the MMAs of Q tile 0 and 1.  An issuing warp runs converged (all lanes compute
+//     tiles, warp 12 issues the MMAs.  It runs converged (all lanes compute
 //     the warp-uniform descriptors, lane 0 executes the tcgen05 instructions): a single
 //     diverged thread was starved of issue slots by the arithmetic-heavy softmax warps that
 //     share its scheduler (measured 100-600 cycles per tcgen05.mma instead of 64).
 //   * Every exponential is one ex2.approx on the special-function unit.  (Evaluating a share of them on the
-//     FMA pipe -- Cody-Waite split + cubic -- was measured at 1/16, 1/8, 1/4 and 1/2 of the scores: the loop is
-//     bound by the number of instructions the softmax warps issue, not by that unit, and every share was slower
-//     than none.)
-//   * The running maximum m is set on a row's first tile and after that only raised when a tile's sum of
+//     FMA pipe -- Cody-Waite split + cubic -- was measured at 1/16, 1/8, 1/4, 3/8 and 1/2 of the scores, with
+//     64-key and with 128-key tiles, and was slower than none at every share.)
+//   * The running maximum m is set on a row's first tile and after that only raised when a half's sum of
 //     2^(score - m) reaches 2^64: the exponentials are taken against m as it stands, with no search for the
-//     tile's maximum first (one instruction per two scores less in a loop bound by issued instructions) and
-//     hardly ever a rescaling of O in tensor memory; (O, m, l) stay consistent whatever m is, so the final
-//     division, or the split merge, needs no correction, and fp32 (sums, O) and bf16 (P) carry the range.
-//   * A long key list can be split across CTAs (blockIdx.z); partial (O, m, l) go to the
-//     context's scratch through coalesced stores, and the CTA that finishes a unit last merges
+//     half's maximum first and hardly ever a rescaling of O in tensor memory; (O, m, l) stay consistent
+//     whatever m is, so the final division, or the split merge, needs no correction, and fp32 (sums, O) and
+//     bf16 (P) carry the range.
+//   * A long key list can be split across CTAs (blockIdx.z); a two-way split runs as CTA pairs that exchange
+//     halves of their partial (O, m, l) through distributed shared memory (PAIR, below); otherwise the partials
+//     go to the context's scratch through coalesced stores, and the CTA that finishes a unit last merges
 //     them with its own accumulator (an arrival counter per unit decides; nobody waits).
+//   * Two-position attention (Section 3.2) is a split by construction: the first half of the splits
+//     covers the list entries of I and M_k with the second encoding (Qg, Kg), the other half covers
+//     L and C with (Q, K), so a CTA holds one pair of Q tiles whichever part it works on, and the
+//     merge that joins key-list splits also joins the two parts (Algorithm 1's merge of (O, m, l)).
 #include <cstring>
 
 #include "esa_internal.h"
@@ -42,9 +47,10 @@ namespace esa {
 
 namespace {
 
-constexpr int TC_BN = 64;             // keys per tile
+constexpr int TC_BN = 128;            // keys per tile
+constexpr int TC_HALF = 64;           // keys per softmax step (half a tile)
 constexpr int TC_ROWS = 256;          // rows per CTA
-constexpr int TC_STAGES = 4;          // K and V tiles in flight
+constexpr int TC_STAGES = 2;          // K tiles and V tiles in shared memory
 constexpr int TC_SOFTMAX_WARPS = 8;
 constexpr int TC_PRODUCER_WARPS = 4;
 constexpr int TC_MMA_WARP = TC_SOFTMAX_WARPS + TC_PRODUCER_WARPS;
@@ -79,6 +85,7 @@ struct TcAttendParams {
     int* unit_count;    // arrivals per (sequence, key/value head, row tile); returns to 0 after each launch
     int q_tma;          // Q tiles arrive by TMA (one arrival) instead of cp.async (one per producer thread)
     int staged;         // the caches hold the attended list itself: row j = list entry j
+    int two;            // two-position attention: splits [0, nsplit/2) take I and M_k with (Qg, Kg), the rest L and C with (Q, K)
     float scale_log2;
     SeqMeta meta;
 };
@@ -90,10 +97,9 @@ enum {
     BAR_V_FULL = BAR_K_FULL + TC_STAGES,    // TC_STAGES
     BAR_K_EMPTY = BAR_V_FULL + TC_STAGES,   // TC_STAGES
     BAR_V_EMPTY = BAR_K_EMPTY + TC_STAGES,  // TC_STAGES
-    BAR_S_READY = BAR_V_EMPTY + TC_STAGES,  // [Q tile][buffer]: 4
-    BAR_P_READY = BAR_S_READY + 4,          // [Q tile][buffer]: 4 (the softmax may run two tiles ahead of
-                                            // the issuing warp, so one barrier per buffer keeps waits adjacent)
-    BAR_PV_DONE = BAR_P_READY + 4,          // per Q tile: 2
+    BAR_S_READY = BAR_V_EMPTY + TC_STAGES,  // per Q tile: 2, one phase per tile
+    BAR_P_READY = BAR_S_READY + 2,          // [Q tile][half]: 4, one phase per tile
+    BAR_PV_DONE = BAR_P_READY + 4,          // per Q tile: 2, one phase per half
     BAR_O_READY = BAR_PV_DONE + 2,          // per Q tile: 2, completes once
     BAR_PAIR = BAR_O_READY + 2,             // PAIR: the partner's half of the partial result has landed; completes once
     BAR_COUNT = BAR_PAIR + 1
@@ -179,10 +185,6 @@ __device__ __forceinline__ void store_half_rows(const float* acc, float4* stage,
     __syncwarp();
 }
 
-// TWO (two-position attention): the list entries of I and M_k take their logits from Qg and Kg, the
-// entries of L and C from Q and K.  Both pairs of Q tiles stay in shared memory (three K/V stages instead
-// of four make room), the I u M_k part of the key list is padded to whole tiles so that a tile never
-// mixes the two, and the issuing warp picks the Q tiles by the tile's part.
 // PAIR: the key list is split in two and the two CTAs of a unit form a thread-block cluster.  CTA r finishes
 // column half r of the unit's rows.  Each parks the other column half of its partial (O, m, l) in its own shared
 // memory (the K/V stages, idle by then); after a cluster barrier (both CTAs have finished their products) each
@@ -192,10 +194,10 @@ __device__ __forceinline__ void store_half_rows(const float* acc, float4* stage,
 // (Measured for the 128 KB of a partial: loads from the other CTA's shared memory 9 us, one 16-byte store per
 // lane and row 6 us, bulk copies 3.5 us.)  A second cluster barrier keeps each sender's shared memory alive until
 // its copies have landed.
-template <int D, bool TWO, bool PAIR>
+template <int D, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap qgmap, TcAttendParams p) {
-    constexpr int STAGES = TWO ? 3 : TC_STAGES;
+    constexpr int STAGES = TC_STAGES;
     constexpr int CH = D / 8;                   // 16-byte chunks per row
     constexpr int Q_TILE_BYTES = 128 * D * 2;   // one 128-row Q tile
     constexpr int Q_BLK_BYTES = 128 * 128;      // one 64-column block of it
@@ -205,8 +207,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem;                               // 2 Q tiles
-    uint8_t* sQg = sQ + 2 * Q_TILE_BYTES;             // 2 more (TWO)
-    uint8_t* sK = sQg + (TWO ? 2 * Q_TILE_BYTES : 0); // STAGES tiles
+    uint8_t* sK = sQ + 2 * Q_TILE_BYTES;              // STAGES tiles
     uint8_t* sV = sK + STAGES * KV_TILE_BYTES;        // STAGES tiles
     __shared__ uint64_t bars[BAR_COUNT];
     __shared__ uint32_t tmem_slot;
@@ -231,14 +232,12 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_K_FULL + s), TC_PRODUCERS);
             mbar_init(bar(BAR_V_FULL + s), TC_PRODUCERS);
-            mbar_init(bar(BAR_K_EMPTY + s), 2);          // one commit per Q tile's issuing warp
-            mbar_init(bar(BAR_V_EMPTY + s), 2);
+            mbar_init(bar(BAR_K_EMPTY + s), 1);          // one commit, after the products of both Q tiles
+            mbar_init(bar(BAR_V_EMPTY + s), 1);
         }
-        for (int s = 0; s < 4; ++s) {                    // [Q tile][buffer]
-            mbar_init(bar(BAR_S_READY + s), 1);
-            mbar_init(bar(BAR_P_READY + s), 128);        // every softmax thread of the tile arrives
-        }
+        for (int s = 0; s < 4; ++s) mbar_init(bar(BAR_P_READY + s), 128);   // every softmax thread of the Q tile arrives
         for (int q = 0; q < 2; ++q) {
+            mbar_init(bar(BAR_S_READY + q), 1);
             mbar_init(bar(BAR_PV_DONE + q), 1);
             mbar_init(bar(BAR_O_READY + q), 1);
         }
@@ -250,7 +249,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
-    // columns: S of Q tile q, buffer u at q * 128 + u * 64; O of Q tile q at 256 + q * D
+    // columns: S of Q tile q at q * 128 (half u at + u * 64); O of Q tile q at 256 + q * D
     // everything read from global memory comes after the preceding kernel (the selection) is complete
     pdl_wait();
     pdl_launch_dependents();
@@ -263,16 +262,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
 
     const int r_last = min(R, row0 + TC_ROWS) - 1;
     const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
-    // tiles: the first far_tiles cover the list entries [0, far_end) of I and M_k (TWO: padded to whole tiles),
-    // the rest the entries from far_end on
-    const int far_end = TWO ? n_glob : 0;
-    const int far_tiles = TWO ? (n_glob + TC_BN - 1) / TC_BN : 0;
-    auto tile_key0 = [&](int T) { return T < far_tiles ? T * TC_BN : far_end + (T - far_tiles) * TC_BN; };
-    const int n_tiles_all = far_tiles + max(0, (j_end - far_end + TC_BN - 1) / TC_BN);
-    const int per = (n_tiles_all + p.nsplit - 1) / p.nsplit;
-    const int tile_begin = split * per;
+    // The part of the key list this CTA's group of splits covers: all of it, or (two-position attention)
+    // the entries of I and M_k for the first half of the splits and those of L and C for the second.
+    const int grp = p.two ? p.nsplit / 2 : p.nsplit;       // splits that share a part
+    const bool far = p.two && split < grp;                 // this CTA works with (Qg, Kg)
+    const int part_lo = (p.two && !far) ? n_glob : 0;
+    const int part_hi = far ? n_glob : j_end;
+    const int s_in = (p.two && !far) ? split - grp : split;
+    const int n_tiles_all = max(0, (part_hi - part_lo + TC_BN - 1) / TC_BN);
+    const int per = (n_tiles_all + grp - 1) / grp;
+    const int tile_begin = s_in * per;
     const int tile_end = min(n_tiles_all, tile_begin + per);
     const int n_tiles = max(0, tile_end - tile_begin);
+    auto tile_key0 = [&](int T) { return part_lo + (tile_begin + T) * TC_BN; };   // first list position of the CTA's T-th tile
 
     if (warp_u < TC_SOFTMAX_WARPS) reg_alloc<TC_REGS_SOFTMAX>();
     else reg_dealloc<TC_REGS_OTHER>();
@@ -284,38 +286,39 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         const int row = row0 + qt * 128 + lane_base + lane;
         const uint32_t tS = tmem_addr(tmem, lane_base, qt * 128);
         const uint32_t tO = tmem_addr(tmem, lane_base, 256 + qt * D);
-        const int lim = c_first + min(row / G, p.l_C - 1) + 1;          // first invisible list position
-        const int lim_min = c_first + min((row0 + qt * 128) / G, p.l_C - 1) + 1;   // smallest limit of the tile
+        // first invisible list position of this row, and the smallest such limit of the Q tile
+        const int lim = min(part_hi, c_first + min(row / G, p.l_C - 1) + 1);
+        const int lim_min = min(part_hi, c_first + min((row0 + qt * 128) / G, p.l_C - 1) + 1);
         const float sl2 = p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
 
-        for (int j = 0; j < n_tiles; ++j) {
-            const int key0 = tile_key0(tile_begin + j);
-            const bool far = tile_begin + j < far_tiles;
-            const int lim_t = far ? far_end : lim;           // first masked list position of this tile for this row
-            const int u = j & 1;
-            mbar_wait(bar(BAR_S_READY + qt * 2 + u), (j >> 1) & 1, wc);
-            tc_fence_after_sync();
-            const bool need_mask = key0 + TC_BN > (far ? far_end : lim_min);
+        for (int j = 0; j < 2 * n_tiles; ++j) {             // j counts halves: tile j >> 1, half j & 1
+            const int T = j >> 1, u = j & 1;
+            const int key0 = tile_key0(T) + u * TC_HALF;
+            if (u == 0) {
+                mbar_wait(bar(BAR_S_READY + qt), T & 1, wc);
+                tc_fence_after_sync();
+            }
+            const bool need_mask = key0 + TC_HALF > lim_min;
             // the score row of this thread: 64 fp32 columns
-            uint32_t v[TC_BN];
+            uint32_t v[TC_HALF];
             tmem_ld32(tS + u * 64, v);
             tmem_ld32(tS + u * 64 + 32, v + 32);
             tmem_wait_ld();
             if (need_mask) {
 #pragma unroll
-                for (int i = 0; i < TC_BN; ++i)
-                    if (key0 + i >= lim_t) v[i] = 0xff800000u;   // -inf
+                for (int i = 0; i < TC_HALF; ++i)
+                    if (key0 + i >= lim) v[i] = 0xff800000u;   // -inf
             }
-            // P = 2^(S * scale - m) as packed bf16 (it will overwrite the first half of the S buffer); returns the sum
-            // of the tile.  A row without a visible key so far has m = -inf: its P must be 0, not 2^(+inf).
-            uint32_t pk[TC_BN / 2];
+            // P = 2^(S * scale - m) as packed bf16 (it will overwrite the first 32 columns of this half); returns the
+            // sum of the half.  A row without a visible key so far has m = -inf: its P must be 0, not 2^(+inf).
+            uint32_t pk[TC_HALF / 2];
             auto exps = [&](float m) {
                 const float neg_m = (m == -INFINITY) ? 0.f : -m;
                 const float2 sl2v = make_float2(sl2, sl2), nm = make_float2(neg_m, neg_m);
                 float2 sum4[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-                for (int i = 0; i < TC_BN / 2; ++i) {
+                for (int i = 0; i < TC_HALF / 2; ++i) {
                     const float2 x = ffma2(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2v, nm);
                     float2 e;
                     e.x = fast_exp2(x.x);
@@ -326,34 +329,34 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 const float2 a = fadd2(sum4[0], sum4[1]), c = fadd2(sum4[2], sum4[3]);
                 return (a.x + a.y) + (c.x + c.y);
             };
-            // The exponentials are taken against the running maximum as it stands, without looking for the tile's
+            // The exponentials are taken against the running maximum as it stands, without looking for the half's
             // own maximum first: (O, m, l) stay consistent whatever m is, and fp32 and bf16 carry the range.  Only when
-            // the tile's sum shows that some score lies far above m (or no key has been seen yet) is the maximum
-            // raised, O rescaled and the tile redone.  The decision is taken per warp: tensor-memory accesses are
+            // the half's sum shows that some score lies far above m (or no key has been seen yet) is the maximum
+            // raised, O rescaled and the half redone.  The decision is taken per warp: tensor-memory accesses are
             // warp-wide.
-            float tile_sum = 0.f;
+            float part_sum = 0.f;
             bool redo = m_run == -INFINITY;
             if (!__any_sync(0xffffffffu, redo)) {
-                tile_sum = exps(m_run);
-                redo = !(tile_sum < kSumLimit);              // also true for inf and NaN
+                part_sum = exps(m_run);
+                redo = !(part_sum < kSumLimit);              // also true for inf and NaN
             }
             if (__any_sync(0xffffffffu, redo)) {
                 float mxc[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) mxc[c] = fmaxf(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
 #pragma unroll
-                for (int i = 16; i < TC_BN; i += 16)
+                for (int i = 16; i < TC_HALF; i += 16)
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         mxc[c] = fmax3(mxc[c], __uint_as_float(v[i + 2 * c]), __uint_as_float(v[i + 2 * c + 1]));
                 const float mx = fmaxf(fmax3(mxc[0], mxc[1], mxc[2]), fmax3(fmax3(mxc[3], mxc[4], mxc[5]), mxc[6], mxc[7]));
                 const float m_new = fmaxf(m_run, mx * sl2);
-                // 0 on a row's first visible tile; a row that has seen no key yet keeps (m, l) = (-inf, 0)
+                // 0 on a row's first visible half; a row that has seen no key yet keeps (m, l) = (-inf, 0)
                 const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m_run - m_new);
                 l_run *= alpha;
                 m_run = m_new;
                 if (j > 0) {
-                    // O must be quiescent: wait for the P V product of the previous tile
+                    // O must be quiescent: wait for the P V product of the previous half
                     mbar_wait(bar(BAR_PV_DONE + qt), (j - 1) & 1, wc);
                     tc_fence_after_sync();
 #pragma unroll
@@ -366,18 +369,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                         tmem_st32(tO + c0, o);
                     }
                 }
-                tile_sum = exps(m_run);
+                part_sum = exps(m_run);
             }
             tmem_st32(tS + u * 64, pk);
-            l_run += tile_sum;
+            l_run += part_sum;
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BAR_P_READY + qt * 2 + u));
         }
 
         // ---- epilogue: O / l  (or the unnormalised partial for the split merge)
-        // (BAR_PV_DONE cannot serve here: a parity wait tells adjacent phases apart only, and this
-        // thread may be two phases behind or level with it; BAR_O_READY completes exactly once.)
+        // (BAR_O_READY completes exactly once.)
         if (n_tiles > 0) {
             mbar_wait(bar(BAR_O_READY + qt), 0, wc);
             tc_fence_after_sync();
@@ -412,10 +414,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             constexpr int NCELL = DH / 4;              // 16-byte cells per half row
             constexpr uint32_t HALF_BYTES = TC_ROWS * DH * 4, ML_BYTES = TC_ROWS * 8;
             const int rl = qt * 128 + lane_base + lane;                       // row within the CTA
-            // K/V stages (TWO: from the second pair of Q tiles on): [0, HALF_BYTES) the half this CTA sends,
+            // K/V stages: [0, HALF_BYTES) the half this CTA sends,
             // [HALF_BYTES, 2 HALF_BYTES) the half it receives; rows of DH fp32, cells XOR-swizzled by the row
-            uint8_t* park = TWO ? sQg : sK;
-            static_assert((TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES >= 2 * HALF_BYTES, "both halves must fit");
+            uint8_t* park = sK;
+            static_assert(2 * STAGES * KV_TILE_BYTES >= 2 * HALF_BYTES, "both halves must fit");
             // both warpgroups have passed their O_READY: no MMA reads the Q tiles or the K/V stages any more
             asm volatile("bar.sync 1, 256;\n" ::: "memory");
             // shared memory of the Q tiles: warp w of Q tile q stages its bf16 result in the first half of the 8 KB
@@ -589,10 +591,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 // their O_READY before the arrival barrier above, so no MMA reads them any more.
                 const int64_t own_off = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D;     // this lane's row of O, in elements
                 const uint32_t own_lo = (uint32_t)own_off, own_hi = (uint32_t)(own_off >> 32);
-                // (TWO: the ring starts at the second pair of Q tiles, idle as well, since three K/V stages alone are too small)
-                constexpr int RING_BYTES = (TWO ? 2 * Q_TILE_BYTES : 0) + 2 * STAGES * KV_TILE_BYTES;
+                constexpr int RING_BYTES = 2 * STAGES * KV_TILE_BYTES;
                 static_assert(RING_BYTES / 8 >= 2 * 32 * (D / 8) * 16, "two buffers of 32 rows x D/2 floats per warp");
-                float4* ring = reinterpret_cast<float4*>((TWO ? sQg : sK) + warp_u * (RING_BYTES / 8));
+                float4* ring = reinterpret_cast<float4*>(sK + warp_u * (RING_BYTES / 8));
                 const int n_other = p.nsplit - 1, n_pairs = 2 * n_other;
                 auto other = [&](int i) { const int s = i % n_other; return s + (s >= split ? 1 : 0); };
                 auto issue = [&](int i) {
@@ -685,27 +686,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
     } else if (warp_u < TC_MMA_WARP) {
         // ------------------------------------------------------------ producers: Q, then K/V tiles
         const int ptid = tid - TC_SOFTMAX_WARPS * 32;      // 0..127
-        const int chunk = ptid % CH;                       // this thread's 16-byte chunk of every row
-        const int rsub = ptid / CH;                        // first row handled
-        constexpr int RSTEP = TC_PRODUCERS / CH;           // rows advanced per iteration
-        const int cin = chunk & 7;
         if (n_tiles > 0 && p.q_tma) {
             // two boxes per 64-column block: rows (query, head-in-group) of one key/value head
             if (ptid == 0) {
-                mbar_arrive_expect_tx(bar(BAR_Q_FULL), (TWO ? 4 : 2) * Q_TILE_BYTES);
+                mbar_arrive_expect_tx(bar(BAR_Q_FULL), 2 * Q_TILE_BYTES);
+                const CUtensorMap* qm = far ? &qgmap : &qmap;
 #pragma unroll
                 for (int qt = 0; qt < 2; ++qt)
 #pragma unroll
-                    for (int blk = 0; blk < D / 64; ++blk) {
-                        tma_load_3d(smem_u32(sQ + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), &qmap, blk * 64, kvh * G,
+                    for (int blk = 0; blk < D / 64; ++blk)
+                        tma_load_3d(smem_u32(sQ + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), qm, blk * 64, kvh * G,
                                     b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
-                        if (TWO)
-                            tma_load_3d(smem_u32(sQg + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), &qgmap, blk * 64, kvh * G,
-                                        b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
-                    }
             }
         } else if (n_tiles > 0) {
             // group sizes that do not divide 128: 16-byte copies, row by row
+            const int chunk = ptid % CH, rsub = ptid / CH, cin = chunk & 7;
+            constexpr int RSTEP = TC_PRODUCERS / CH;
+            const __nv_bfloat16* Qsrc = far ? p.Qg : p.Q;
             for (int r = rsub; r < TC_ROWS; r += RSTEP) {
                 const int row = row0 + r;
                 const bool ok = row < R;
@@ -713,21 +710,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 const int64_t qoff = (((int64_t)b * p.l_C + cq) * p.H + kvh * G + g) * D + chunk * 8;
                 const int rr = r & 127;
                 const uint32_t doff = (r >> 7) * Q_TILE_BYTES + (chunk >> 3) * Q_BLK_BYTES + rr * 128 + ((cin ^ (rr & 7)) << 4);
-                cp_async16(sQ + doff, p.Q + qoff, ok ? 16 : 0);
-                if (TWO) cp_async16(sQg + doff, p.Qg + qoff, ok ? 16 : 0);
+                cp_async16(sQ + doff, Qsrc + qoff, ok ? 16 : 0);
             }
             cp_async_arrive_noinc(bar(BAR_Q_FULL));
         }
         // K/V tiles: four threads share a row (one instruction of the four covers 64 contiguous bytes of it: whole
-        // sectors), so a thread works out the cache position of two rows per tile, not of eight, and copies CH / 4
-        // chunks of each; the loop is bound by the instructions the CTA's warps issue, these included.
+        // sectors), so a thread works out the cache position of four rows per 128-key tile, not of sixteen, and
+        // copies CH / 4 chunks of each; the loop is sensitive to the instructions the CTA's warps issue, these included.
         constexpr int TPR = 4;                             // threads per row
         constexpr int RPP = TC_PRODUCERS / TPR;            // rows per pass: 32
-        constexpr int NPASS = TC_BN / RPP;                 // 2
+        constexpr int NPASS = TC_BN / RPP;                 // 4
         constexpr int CPT = CH / TPR;                      // chunks per thread and row: 4 (D = 128) or 2
         const int q4 = ptid % TPR, rfirst = ptid / TPR;
-        const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
-        const __nv_bfloat16* Kgb = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
+        const __nv_bfloat16* Kb = (far ? p.Kg : p.K) + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
@@ -738,14 +733,12 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             const int r = rfirst + it * RPP;
             row_off[it] = (uint32_t)(r * 128) | (uint32_t)((r & 7) << 4);      // XOR with (c & 7) << 4 gives the swizzled chunk
         }
+        const int row_lim = far ? part_hi : n_att;          // list positions of this CTA's part end here
         int bad_idx = 0;
         for (int j = 0; j < n_tiles; ++j) {
             const int s = j % STAGES;
             const uint32_t ph = ((j / STAGES) & 1) ^ 1;
-            const int key0 = tile_key0(tile_begin + j);
-            const bool far = tile_begin + j < far_tiles;
-            const int row_lim = far ? far_end : n_att;      // list positions of this tile end here
-            const __nv_bfloat16* Ksrc = far ? Kgb : Kb;
+            const int key0 = tile_key0(j);
             int pos[NPASS];
             uint32_t from_idx = 0;                      // rows whose position was read from the selection
 #pragma unroll
@@ -768,7 +761,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 if ((from_idx >> it) & 1u) pos[it] = clamp_selected(pos[it], i_end, m_end, bad_idx);
 #pragma unroll
             for (int it = 0; it < NPASS; ++it) {
-                const __nv_bfloat16* src = Ksrc + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
+                const __nv_bfloat16* src = Kb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
                 const int nbytes = pos[it] < 0 ? 0 : 16;
                 uint8_t* tile = sK + s * KV_TILE_BYTES;
 #pragma unroll
@@ -794,61 +787,69 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         }
         if (bad_idx) atomicExch(p.status, kStatusBadIndex);
         cp_async_wait<0>();
-    } else if (warp_u < TC_MMA_WARP + 2 && n_tiles > 0) {
-        // ------------------------------------------------------------ MMA issue: one converged warp per Q tile,
-        // lane 0 leads.  Two warps halve the chain of waits and commits that sits between batches of MMAs
-        // (the tensor core's queue is too shallow to hide it); their products interleave freely because the
-        // Q tiles share nothing but read-only K/V tiles.
-        const int qt = warp_u - TC_MMA_WARP;
+    } else if (warp_u == TC_MMA_WARP && n_tiles > 0) {
+        // ------------------------------------------------------------ MMA issue: one converged warp, lane 0 leads.
+        // The fixed order (Q tile 0's products of a tile, then Q tile 1's) keeps the two Q tiles half a period
+        // apart: S of Q tile 1 always becomes ready one block of products after S of Q tile 0, so each softmax
+        // warpgroup computes while the tensor core works for the other one.  (Two independent issuing warps settle
+        // into lockstep instead: both softmaxes, then both blocks.)
         const uint32_t lead = lane == 0;
         constexpr uint32_t ID_QK = idesc_bf16(128, TC_BN, false, false);
         constexpr uint32_t ID_PV = idesc_bf16(128, D, false, true);
         const uint32_t hi = desc_hi_sw128();
-        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ)) + qt * (Q_TILE_BYTES >> 4);
-        const uint32_t qglo = desc_lo_kmajor(smem_u32(sQg)) + qt * (Q_TILE_BYTES >> 4);
+        const uint32_t qlo = desc_lo_kmajor(smem_u32(sQ));
         const uint32_t klo = desc_lo_kmajor(smem_u32(sK)), vlo = desc_lo_mnmajor(smem_u32(sV), KV_BLK_BYTES);
-        const uint32_t dS = tmem + qt * 128, dO = tmem + 256 + qt * D;
         // descriptor low words advance by compile-time constants (bytes >> 4)
-        auto issue_qk = [&](int s, int u, int j) {          // S[u] = Q . K[s]^T for the CTA's j-th tile
+        auto issue_qk = [&](int qt, int s) {                // S[qt] = Q[qt] . K[s]^T, 128 keys
+            const uint32_t a0 = qlo + qt * (Q_TILE_BYTES >> 4);
             const uint32_t b0 = klo + s * (KV_TILE_BYTES >> 4);
-            const uint32_t qsel = (TWO && tile_begin + j < far_tiles) ? qglo : qlo;
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks)
-                umma_ss(dS + u * 64, qsel + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
+                umma_ss(tmem + qt * 128, a0 + (((ks >> 2) * Q_BLK_BYTES + (ks & 3) * 32) >> 4),
                         b0 + (((ks >> 2) * KV_BLK_BYTES + (ks & 3) * 32) >> 4), hi, ID_QK, ks, lead);
         };
-        auto issue_pv = [&](int s, int u, int acc) {         // O (+)= P[u] . V[s]
-            const uint32_t b0 = vlo + s * (KV_TILE_BYTES >> 4);
+        auto issue_pv = [&](int qt, int s, int u, int acc) { // O[qt] (+)= P[qt][half u] . V[s][keys of half u]
+            const uint32_t b0 = vlo + s * (KV_TILE_BYTES >> 4) + u * ((TC_HALF * 128) >> 4);
 #pragma unroll
-            for (int ks = 0; ks < TC_BN / 16; ++ks)
-                umma_ts(dO, dS + u * 64 + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks, lead);
+            for (int ks = 0; ks < TC_HALF / 16; ++ks)
+                umma_ts(tmem + 256 + qt * D, tmem + qt * 128 + u * 64 + ks * 8, b0 + ks * (2048 >> 4), hi, ID_PV, acc | ks, lead);
         };
         mbar_wait(bar(BAR_Q_FULL), 0, wc);
-        for (int j = 0; j < 2 && j < n_tiles; ++j) {          // scores of the first two tiles
-            mbar_wait(bar(BAR_K_FULL + j), 0, wc);
+        mbar_wait(bar(BAR_K_FULL + 0), 0, wc);
+        fence_async_smem();
+        tc_fence_after_sync();
+        issue_qk(0, 0);
+        umma_commit(bar(BAR_S_READY + 0), lead);
+        issue_qk(1, 0);
+        umma_commit(bar(BAR_S_READY + 1), lead);
+        umma_commit(bar(BAR_K_EMPTY + 0), lead);
+        for (int T = 0; T < n_tiles; ++T) {
+            const int s = T % STAGES;
+            const int Tn = T + 1, sn = Tn % STAGES;
+            const bool more = Tn < n_tiles;
+            mbar_wait(bar(BAR_V_FULL + s), (T / STAGES) & 1, wc);
             fence_async_smem();
-            tc_fence_after_sync();
-            issue_qk(j, j, j);
-            umma_commit(bar(BAR_S_READY + qt * 2 + j), lead);
-            umma_commit(bar(BAR_K_EMPTY + j), lead);
-        }
-        for (int j = 0; j < n_tiles; ++j) {
-            const int s = j % STAGES, u = j & 1;
-            const int jn = j + 2, sn = jn % STAGES;
-            const bool more = jn < n_tiles;
-            mbar_wait(bar(BAR_V_FULL + s), (j / STAGES) & 1, wc);
-            if (more) mbar_wait(bar(BAR_K_FULL + sn), (jn / STAGES) & 1, wc);
-            fence_async_smem();
-            mbar_wait(bar(BAR_P_READY + qt * 2 + u), (j >> 1) & 1, wc);
-            tc_fence_after_sync();
-            issue_pv(s, u, j > 0);
-            umma_commit(bar(BAR_PV_DONE + qt), lead);
-            if (j + 1 == n_tiles) umma_commit(bar(BAR_O_READY + qt), lead);
-            umma_commit(bar(BAR_V_EMPTY + s), lead);
-            if (more) {
-                issue_qk(sn, u, jn);          // reuses buffer u after the P V product above, in issue order
-                umma_commit(bar(BAR_S_READY + qt * 2 + u), lead);
-                umma_commit(bar(BAR_K_EMPTY + sn), lead);
+#pragma unroll
+            for (int qt = 0; qt < 2; ++qt) {
+                mbar_wait(bar(BAR_P_READY + qt * 2 + 0), T & 1, wc);
+                tc_fence_after_sync();
+                issue_pv(qt, s, 0, T > 0);
+                umma_commit(bar(BAR_PV_DONE + qt), lead);
+                if (more && qt == 0) {
+                    mbar_wait(bar(BAR_K_FULL + sn), (Tn / STAGES) & 1, wc);
+                    fence_async_smem();
+                }
+                mbar_wait(bar(BAR_P_READY + qt * 2 + 1), T & 1, wc);
+                tc_fence_after_sync();
+                issue_pv(qt, s, 1, 1);
+                umma_commit(bar(BAR_PV_DONE + qt), lead);
+                if (!more) umma_commit(bar(BAR_O_READY + qt), lead);
+                if (qt == 1) umma_commit(bar(BAR_V_EMPTY + s), lead);
+                if (more) {
+                    issue_qk(qt, sn);         // overwrites S and P of this tile after the P V products above, in issue order
+                    umma_commit(bar(BAR_S_READY + qt), lead);
+                    if (qt == 1) umma_commit(bar(BAR_K_EMPTY + sn), lead);
+                }
             }
         }
     }
@@ -867,17 +868,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
 
 }  // namespace
 
-template <int D, bool TWO, bool PAIR>
+template <int D, bool PAIR>
 static cudaError_t launch_tc_kernel(esa_ctx* ctx, const CUtensorMap& qmap, const CUtensorMap& qgmap, const TcAttendParams& p,
                                     dim3 grid, cudaStream_t st, bool probe_only) {
-    constexpr int smem = (TWO ? 4 : 2) * 128 * D * 2 + 2 * (TWO ? 3 : TC_STAGES) * TC_BN * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D, TWO, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    constexpr int smem = 2 * 128 * D * 2 + 2 * TC_STAGES * TC_BN * D * 2 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(attend_tc_kernel<D, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     // the in-kernel register split assumes the launch allocation it was sized for
     static int regs_checked = 0;
     if (!regs_checked) {
         cudaFuncAttributes fa;
-        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D, TWO, PAIR>);
+        e = cudaFuncGetAttributes(&fa, attend_tc_kernel<D, PAIR>);
         if (e != cudaSuccess) return e;
         if (fa.numRegs != TC_REGS_LAUNCH) return cudaErrorInvalidConfiguration;
         regs_checked = 1;
@@ -899,46 +900,54 @@ static cudaError_t launch_tc_kernel(esa_ctx* ctx, const CUtensorMap& qmap, const
     if (probe_only) {
         // can the device place a pair of these CTAs at all?
         int n_clusters = 0;
-        e = cudaOccupancyMaxActiveClusters(&n_clusters, attend_tc_kernel<D, TWO, PAIR>, &cfg);
+        e = cudaOccupancyMaxActiveClusters(&n_clusters, attend_tc_kernel<D, PAIR>, &cfg);
         if (e != cudaSuccess) return e;
         return n_clusters > 0 ? cudaSuccess : cudaErrorNotSupported;
     }
-    return cudaLaunchKernelEx(&cfg, attend_tc_kernel<D, TWO, PAIR>, qmap, qgmap, p);
+    return cudaLaunchKernelEx(&cfg, attend_tc_kernel<D, PAIR>, qmap, qgmap, p);
 }
 
-template <int D, bool TWO>
+template <int D>
 static cudaError_t launch_tc(esa_ctx* ctx, TcAttendParams& p, int B, int n_att_max, cudaStream_t st, int* nsplit_out) {
     const int R = p.l_C * p.G;
     const int row_tiles = (R + TC_ROWS - 1) / TC_ROWS;
     p.Rp = (R + 1) & ~1;
     if ((size_t)B * p.HG * row_tiles > ctx->att_count_elems) return cudaErrorNotSupported;
     // Split the key list when that fills the machine better: cost model = waves x tiles per CTA
-    // (+1 tile-equivalent of fixed work per CTA), one CTA per SM.
+    // (+ half a tile-equivalent of fixed work per CTA), one CTA per SM.  Two-position attention needs an even
+    // number of splits (one group per part); its longer part sets the tiles per CTA.
     const int ctas = row_tiles * p.HG * B;
-    const int n_tiles = (n_att_max + TC_BN - 1) / TC_BN + (TWO ? 1 : 0);
-    int best = 1;
+    const int n_tiles = (n_att_max + TC_BN - 1) / TC_BN;
+    int i_end_max = 0;
+    for (int b = 0; b < B; ++b) i_end_max = max(i_end_max, p.meta.i_end[b]);
+    const int far_tiles = min(n_tiles, (i_end_max + p.top_k + TC_BN - 1) / TC_BN);
+    const int step = p.two ? 2 : 1;
+    int best = 0;
     double best_cost = 1e30;
-    for (int ns = 1; ns <= kAttPrefillSplits && ns <= n_tiles; ++ns) {
+    for (int ns = step; ns <= kAttPrefillSplits && (ns <= n_tiles || best == 0); ns += step) {
         if ((size_t)B * p.HG * ns * p.Rp * (D + 2) > ctx->att_part_elems) break;
-        const int per = (n_tiles + ns - 1) / ns;
+        const int grp = p.two ? ns / 2 : ns;
+        const int longest = p.two ? max(far_tiles, n_tiles - far_tiles + 1) : n_tiles;
+        const int per = (longest + grp - 1) / grp;
         const int waves = (ctas * ns + ctx->num_sms - 1) / ctx->num_sms;
-        const double cost = (double)waves * (per + 1.0) + (ns > 1 ? 0.5 * ns : 0.0);
+        const double cost = (double)waves * (per + 0.5) + (ns > 1 ? 0.25 * ns : 0.0);
         if (cost < best_cost - 1e-9) { best_cost = cost; best = ns; }
     }
+    if (best == 0) return cudaErrorNotSupported;
     p.nsplit = best;
     *nsplit_out = best;
     CUtensorMap qmap, qgmap;
     p.q_tma = make_tensor_map_q(&qmap, p.Q, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
-    if (p.q_tma && TWO) p.q_tma = make_tensor_map_q(&qgmap, p.Qg, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
+    if (p.q_tma && p.two) p.q_tma = make_tensor_map_q(&qgmap, p.Qg, (uint64_t)B * p.l_C, p.H, D, p.G) ? 1 : 0;
     if (!p.q_tma) memset(&qmap, 0, sizeof(qmap));
-    if (!p.q_tma || !TWO) memset(&qgmap, 0, sizeof(qgmap));
+    if (!p.q_tma || !p.two) memset(&qgmap, 0, sizeof(qgmap));
     const dim3 grid(row_tiles, p.HG, B * best);
     // a two-way split runs as CTA pairs that merge through distributed shared memory, where the device can place pairs
     static int pair_ok = -1;                                 // per instantiation; probed once
-    if (best == 2 && pair_ok < 0) pair_ok = launch_tc_kernel<D, TWO, true>(ctx, qmap, qgmap, p, grid, st, true) == cudaSuccess ? 1 : 0;
+    if (best == 2 && pair_ok < 0) pair_ok = launch_tc_kernel<D, true>(ctx, qmap, qgmap, p, grid, st, true) == cudaSuccess ? 1 : 0;
     ProfScope prof(ctx, KC_ATTEND_TC, st);
-    cudaError_t e = (best == 2 && pair_ok == 1) ? launch_tc_kernel<D, TWO, true>(ctx, qmap, qgmap, p, grid, st, false)
-                                                : launch_tc_kernel<D, TWO, false>(ctx, qmap, qgmap, p, grid, st, false);
+    cudaError_t e = (best == 2 && pair_ok == 1) ? launch_tc_kernel<D, true>(ctx, qmap, qgmap, p, grid, st, false)
+                                                : launch_tc_kernel<D, false>(ctx, qmap, qgmap, p, grid, st, false);
     ctx->launches += 1;
     return e;
 }
@@ -955,12 +964,13 @@ cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* 
     p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.status = ctx->status;
     p.unit_count = ctx->att_count;
     p.staged = staged ? 1 : 0;
+    p.two = two ? 1 : 0;
     p.max_tokens = cache_rows > 0 ? cache_rows : ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
     p.meta = meta;
-    if (ctx->d == 128) return two ? launch_tc<128, true>(ctx, p, B, n_att_max, st, nsplit_out) : launch_tc<128, false>(ctx, p, B, n_att_max, st, nsplit_out);
-    if (ctx->d == 64) return two ? launch_tc<64, true>(ctx, p, B, n_att_max, st, nsplit_out) : launch_tc<64, false>(ctx, p, B, n_att_max, st, nsplit_out);
+    if (ctx->d == 128) return launch_tc<128>(ctx, p, B, n_att_max, st, nsplit_out);
+    if (ctx->d == 64) return launch_tc<64>(ctx, p, B, n_att_max, st, nsplit_out);
     return cudaErrorNotSupported;
 }
 
