@@ -397,19 +397,20 @@ attend_decode_kernel(AttendParams p) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     uint4* ring = dec_smem + warp * (DEC_STAGES * STAGE_CHUNKS);
-    pdl_wait();
-    pdl_launch_dependents();
 
+    // The rows of L that are older than this step's token do not depend on the selection, nor on anything the
+    // preceding kernels of the step wrote: every CTA attends its share of them BEFORE the wait for the preceding
+    // kernel (phase 0, positions counted within L u C: cache row m_end + u), while the selection kernel is
+    // still at work on a handful of SMs, and its share of the rest of the list after it (phase 1, list positions).
+    // (Not with two position encodings, nor when the caches hold the staged list: phase 1 alone does everything.)
     const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
-    int n_sel = p.n_sel[b];
-    n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
-    const int n_glob = i_end + n_sel;
-    const int n_att = n_glob + (t - m_end) + 1;            // the single query sees every listed key
-
-    // this CTA's part of the key list, in whole iterations of one warp
-    const int iters_all = (n_att + DEC_ROWS - 1) / DEC_ROWS;
-    const int per = (iters_all + p.nsplit - 1) / p.nsplit;
-    const int it_begin = split * per, it_end = min(iters_all, it_begin + per);
+    const bool early = !TWO && !p.staged;
+    const int u_pre = early ? ((t - m_end) / DEC_ROWS) * DEC_ROWS : 0;     // rows of L done in phase 0: whole iterations
+    const int itA_all = u_pre / DEC_ROWS;
+    const int perA = (itA_all + p.nsplit - 1) / p.nsplit;
+    const int itA_begin = min(itA_all, split * perA), itA_end = min(itA_all, itA_begin + perA);
+    // phase 1, set after the wait
+    int n_glob = 0, n_att = 0, itF = 0, itT = 0;
 
     const int my_chunk = lane % CH, my_row = lane / CH;     // copies of this lane: rows my_row + i * ROWS_PER_PASS
     const __nv_bfloat16* Kb = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + my_chunk * 8;
@@ -418,26 +419,35 @@ attend_decode_kernel(AttendParams p) {
     const int32_t* idx = p.idx + (int64_t)b * p.top_k;
     const int64_t tok_stride = (int64_t)p.HG * D;
 
-    // list positions -> token positions of the rows of iteration `it` that this lane copies
+    // Phase 1 walks the iterations (16 list positions each) that still hold a row to attend: those below
+    // itF = ceil(n_glob / 16) (I and M_k) and those from itT on (the rows of L u C left for this phase).
+    auto iter_of = [&](int ph, int v) { return (ph == 0 || v < itF) ? v : itT + (v - itF); };
+    auto row_valid = [&](int ph, int j) { return ph == 0 || (j < n_att && !(j >= n_glob && j < n_glob + u_pre)); };
+
+    // list positions -> token positions of the rows of iteration `v` that this lane copies
     // (a position read from the selection is range-checked when it is used, one iteration later, so that
     // the index load stays in flight meanwhile; sel_mask remembers which rows those are)
     int bad_idx = 0;
     uint32_t sel_mask = 0;          // rows of the positions looked up last that came from the selection
     uint32_t far_mask = 0;          // rows of the positions looked up last that belong to I or M_k (TWO: their keys come from Kg)
-    auto lookup = [&](int it, int (&pos)[PER_LANE]) {
+    auto lookup = [&](int ph, int v, int v_end, int (&pos)[PER_LANE]) {
         sel_mask = 0;
         far_mask = 0;
+        const int it = iter_of(ph, v);
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) {
             const int j = it * DEC_ROWS + my_row + i * ROWS_PER_PASS;
-            if (TWO && j < n_glob) far_mask |= 1u << i;
             int q = -1;
-            if (it < it_end && j < n_att) {
-                if (p.staged || j < i_end) q = j;
-                else if (j < n_glob) {
-                    q = __ldg(idx + (j - i_end));
-                    sel_mask |= 1u << i;
-                } else q = m_end + (j - n_glob);
+            if (v < v_end) {
+                if (ph == 0) q = m_end + j;
+                else if (row_valid(1, j)) {
+                    if (TWO && j < n_glob) far_mask |= 1u << i;
+                    if (p.staged || j < i_end) q = j;
+                    else if (j < n_glob) {
+                        q = __ldg(idx + (j - i_end));
+                        sel_mask |= 1u << i;
+                    } else q = m_end + (j - n_glob);
+                }
             }
             pos[i] = q;
         }
@@ -483,95 +493,121 @@ attend_decode_kernel(AttendParams p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) o_acc[i][j] = 0.f;
 
-    // prologue: DEC_STAGES - 1 iterations in flight, positions of one more in registers
-    int pos_next[PER_LANE];
-    const int it0 = it_begin + warp;
-#pragma unroll
-    for (int s = 0; s < DEC_STAGES - 1; ++s) {
-        lookup(it0 + s * DEC_WARPS, pos_next);
-        issue(s, pos_next, sel_mask, far_mask);
-        cp_async_commit();
-    }
-    lookup(it0 + (DEC_STAGES - 1) * DEC_WARPS, pos_next);
-
-    int n = 0;
-    for (int it = it0; it < it_end; it += DEC_WARPS, ++n) {
-        issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next, sel_mask, far_mask);
-        cp_async_commit();
-        lookup(it + DEC_STAGES * DEC_WARPS, pos_next);
-        cp_async_wait<DEC_STAGES - 1>();
-        __syncwarp();
-        const uint4* tk = ring + (n % DEC_STAGES) * STAGE_CHUNKS;
-        const uint4* tv = tk + TILE_CHUNKS;
-
-        // S^T[key, head] = K Q^T
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-            uint32_t a[4];
-            load_a_frag<CH>(a, tk, 0, ks * 2, lane);
-            mma_bf16_16816(sc, a, qb[ks][0], qb[ks][1]);
+#pragma unroll 1
+    for (int ph = 0; ph < 2; ++ph) {
+        int v_begin, v_end;
+        if (ph == 0) {
+            v_begin = itA_begin;
+            v_end = itA_end;
+        } else {
+            // everything the selection wrote (n_sel, idx), and rows that may have been appended by the kernel before
+            pdl_wait();
+            pdl_launch_dependents();
+            int n_sel = p.n_sel[b];
+            n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
+            n_glob = i_end + n_sel;
+            n_att = n_glob + (t - m_end) + 1;            // the single query sees every listed key
+            const int iters_all = (n_att + DEC_ROWS - 1) / DEC_ROWS;
+            itF = (n_glob + DEC_ROWS - 1) / DEC_ROWS;
+            itT = max(itF, (n_glob + u_pre) / DEC_ROWS);
+            const int v_all = itF + max(0, iters_all - itT);
+            const int per = (v_all + p.nsplit - 1) / p.nsplit;
+            v_begin = min(v_all, split * per);
+            v_end = min(v_all, v_begin + per);
         }
-        // rows lane / 4 and + 8 of the tile; list positions past the end are masked
-        const int key_lo = it * DEC_ROWS + (lane >> 2);
-        if (TWO && it * DEC_ROWS < n_glob) {
-            // rows of I and M_k: logits against the other query encoding (uniform branch over the warp)
-            float sg[4] = {0.f, 0.f, 0.f, 0.f};
+        // prologue: DEC_STAGES - 1 iterations in flight, positions of one more in registers
+        int pos_next[PER_LANE];
+        const int v0 = v_begin + warp;
 #pragma unroll
+        for (int s = 0; s < DEC_STAGES - 1; ++s) {
+            lookup(ph, v0 + s * DEC_WARPS, v_end, pos_next);
+            issue(s, pos_next, sel_mask, far_mask);
+            cp_async_commit();
+        }
+        lookup(ph, v0 + (DEC_STAGES - 1) * DEC_WARPS, v_end, pos_next);
+
+        int n = 0;
+        for (int v = v0; v < v_end; v += DEC_WARPS, ++n) {
+            issue((n + DEC_STAGES - 1) % DEC_STAGES, pos_next, sel_mask, far_mask);
+            cp_async_commit();
+            lookup(ph, v + DEC_STAGES * DEC_WARPS, v_end, pos_next);
+            cp_async_wait<DEC_STAGES - 1>();
+            __syncwarp();
+            const uint4* tk = ring + (n % DEC_STAGES) * STAGE_CHUNKS;
+            const uint4* tv = tk + TILE_CHUNKS;
+
+            // S^T[key, head] = K Q^T
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 uint32_t a[4];
                 load_a_frag<CH>(a, tk, 0, ks * 2, lane);
-                mma_bf16_16816(sg, a, qbg[ks][0], qbg[ks][1]);
+                mma_bf16_16816(sc, a, qb[ks][0], qb[ks][1]);
             }
-            if (key_lo < n_glob) { sc[0] = sg[0]; sc[1] = sg[1]; }
-            if (key_lo + 8 < n_glob) { sc[2] = sg[2]; sc[3] = sg[3]; }
-        }
-        const bool ok_lo = key_lo < n_att, ok_hi = key_lo + 8 < n_att;
-        sc[0] = ok_lo ? sc[0] * p.scale_log2 : -INFINITY;
-        sc[1] = ok_lo ? sc[1] * p.scale_log2 : -INFINITY;
-        sc[2] = ok_hi ? sc[2] * p.scale_log2 : -INFINITY;
-        sc[3] = ok_hi ? sc[3] * p.scale_log2 : -INFINITY;
-        float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
-        }
-        const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
-        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        if (mn0 != m_run[0] || mn1 != m_run[1]) {          // uniform over the lanes that share the heads
-            const float al0 = fast_exp2(m_run[0] - ms0), al1 = fast_exp2(m_run[1] - ms1);
-            l_run[0] *= al0;
-            l_run[1] *= al1;
-#pragma unroll
-            for (int i = 0; i < D / 16; ++i) {
-                o_acc[i][0] *= al0; o_acc[i][1] *= al1; o_acc[i][2] *= al0; o_acc[i][3] *= al1;
+            // rows lane / 4 and + 8 of the tile; list positions past the end are masked
+            const int it = iter_of(ph, v);
+            const int key_lo = it * DEC_ROWS + (lane >> 2);
+            if (TWO && it * DEC_ROWS < n_glob) {
+                // rows of I and M_k: logits against the other query encoding (uniform branch over the warp)
+                float sg[4] = {0.f, 0.f, 0.f, 0.f};
+    #pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    uint32_t a[4];
+                    load_a_frag<CH>(a, tk, 0, ks * 2, lane);
+                    mma_bf16_16816(sg, a, qbg[ks][0], qbg[ks][1]);
+                }
+                if (key_lo < n_glob) { sc[0] = sg[0]; sc[1] = sg[1]; }
+                if (key_lo + 8 < n_glob) { sc[2] = sg[2]; sc[3] = sg[3]; }
             }
-            m_run[0] = mn0;
-            m_run[1] = mn1;
+            const bool ok_lo = row_valid(ph, key_lo), ok_hi = row_valid(ph, key_lo + 8);
+            sc[0] = ok_lo ? sc[0] * p.scale_log2 : -INFINITY;
+            sc[1] = ok_lo ? sc[1] * p.scale_log2 : -INFINITY;
+            sc[2] = ok_hi ? sc[2] * p.scale_log2 : -INFINITY;
+            sc[3] = ok_hi ? sc[3] * p.scale_log2 : -INFINITY;
+            float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+    #pragma unroll
+            for (int o = 4; o < 32; o <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+            }
+            const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+            const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+            if (mn0 != m_run[0] || mn1 != m_run[1]) {          // uniform over the lanes that share the heads
+                const float al0 = fast_exp2(m_run[0] - ms0), al1 = fast_exp2(m_run[1] - ms1);
+                l_run[0] *= al0;
+                l_run[1] *= al1;
+    #pragma unroll
+                for (int i = 0; i < D / 16; ++i) {
+                    o_acc[i][0] *= al0; o_acc[i][1] *= al1; o_acc[i][2] *= al0; o_acc[i][3] *= al1;
+                }
+                m_run[0] = mn0;
+                m_run[1] = mn1;
+            }
+            const float p0 = fast_exp2(sc[0] - ms0), p1 = fast_exp2(sc[1] - ms1);
+            const float p2 = fast_exp2(sc[2] - ms0), p3 = fast_exp2(sc[3] - ms1);
+            l_run[0] += p0 + p2;
+            l_run[1] += p1 + p3;
+            // P^T as the B operand (k = key, n = head): thread T needs keys 2 (T & 3), +1 (and + 8) of head T / 4;
+            // in the accumulator layout those sit in lanes (key & 7) * 4 + head / 2, packed per head pair.
+            const uint32_t w_lo = pack_bf16(p0, p1), w_hi = pack_bf16(p2, p3);       // keys r and r + 8, heads 2q, 2q + 1
+            const int src0 = (2 * (lane & 3)) * 4 + (lane >> 3), src1 = src0 + 4;
+            const uint32_t a_lo = __shfl_sync(0xffffffffu, w_lo, src0), b_lo = __shfl_sync(0xffffffffu, w_lo, src1);
+            const uint32_t a_hi = __shfl_sync(0xffffffffu, w_hi, src0), b_hi = __shfl_sync(0xffffffffu, w_hi, src1);
+            const uint32_t sel = ((lane >> 2) & 1) ? 0x7632u : 0x5410u;               // odd head: upper halves, else lower
+            const uint32_t pb0 = __byte_perm(a_lo, b_lo, sel), pb1 = __byte_perm(a_hi, b_hi, sel);
+            // O^T[d, head] += V^T P^T: A = V^T from the row-major V tile through transposing ldmatrix
+    #pragma unroll
+            for (int dt = 0; dt < D / 16; ++dt) {
+                uint32_t av[4];
+                const int r = (lane & 7) + ((lane >> 4) & 1) * 8;          // key row of this lane's matrix
+                const int c = dt * 2 + ((lane >> 3) & 1);                 // 16-byte chunk: d 0-7 or 8-15 of the tile
+                ldmatrix_x4_trans(av, tv + swz<CH>(r, c));
+                mma_bf16_16816(o_acc[dt], av, pb0, pb1);
+            }
+            __syncwarp();          // the stage is free for the copy issued next iteration
         }
-        const float p0 = fast_exp2(sc[0] - ms0), p1 = fast_exp2(sc[1] - ms1);
-        const float p2 = fast_exp2(sc[2] - ms0), p3 = fast_exp2(sc[3] - ms1);
-        l_run[0] += p0 + p2;
-        l_run[1] += p1 + p3;
-        // P^T as the B operand (k = key, n = head): thread T needs keys 2 (T & 3), +1 (and + 8) of head T / 4;
-        // in the accumulator layout those sit in lanes (key & 7) * 4 + head / 2, packed per head pair.
-        const uint32_t w_lo = pack_bf16(p0, p1), w_hi = pack_bf16(p2, p3);       // keys r and r + 8, heads 2q, 2q + 1
-        const int src0 = (2 * (lane & 3)) * 4 + (lane >> 3), src1 = src0 + 4;
-        const uint32_t a_lo = __shfl_sync(0xffffffffu, w_lo, src0), b_lo = __shfl_sync(0xffffffffu, w_lo, src1);
-        const uint32_t a_hi = __shfl_sync(0xffffffffu, w_hi, src0), b_hi = __shfl_sync(0xffffffffu, w_hi, src1);
-        const uint32_t sel = ((lane >> 2) & 1) ? 0x7632u : 0x5410u;               // odd head: upper halves, else lower
-        const uint32_t pb0 = __byte_perm(a_lo, b_lo, sel), pb1 = __byte_perm(a_hi, b_hi, sel);
-        // O^T[d, head] += V^T P^T: A = V^T from the row-major V tile through transposing ldmatrix
-#pragma unroll
-        for (int dt = 0; dt < D / 16; ++dt) {
-            uint32_t av[4];
-            const int r = (lane & 7) + ((lane >> 4) & 1) * 8;          // key row of this lane's matrix
-            const int c = dt * 2 + ((lane >> 3) & 1);                 // 16-byte chunk: d 0-7 or 8-15 of the tile
-            ldmatrix_x4_trans(av, tv + swz<CH>(r, c));
-            mma_bf16_16816(o_acc[dt], av, pb0, pb1);
-        }
-        __syncwarp();          // the stage is free for the copy issued next iteration
+        cp_async_wait<0>();
+        __syncwarp();
     }
     cp_async_wait<0>();
     if (bad_idx && p.status) atomicExch(p.status, kStatusBadIndex);

@@ -539,8 +539,8 @@ def test_two_position_attention_llama_shape_and_group_of_seven():
                                                ("c1", 300, 128, None), ("c2", 8192, 512, None), ("c2", 9000, 1, None)])
 def test_attention_with_host_resident_kv(name, t, l_C, n_sel):
     """The K/V cache lives in pinned host memory; the attended rows are staged on the device by the
-    library's gather kernel.  Same bits as esa_attend on device-resident copies, and within the
-    attention tolerance of the oracle."""
+    library's gather kernel.  Same bits as esa_attend on device-resident copies (for a single query: up to a
+    rounding step, the order of the sums differs), and within the attention tolerance of the oracle."""
     cfg = syn.get_config(name)
     p = hp.oracle_params(cfg)
     n = t + l_C
@@ -565,7 +565,16 @@ def test_attention_with_host_resident_kv(name, t, l_C, n_sel):
     O_dev = torch.empty_like(Q)
     ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O_dev, sync=True)
     assert ctx.last_device_status() == 0
-    assert torch.equal(O_host, O_dev)
+    if l_C == 1:
+        # the decode kernel attends the older rows of L ahead of the rest when the caches are indexed by token, and
+        # the whole list in order when they hold the staged rows: the same sums in another order, so the two
+        # results may differ by the rounding of P and of the result (P is rounded to bf16 against the running maximum
+        # of the moment): a bf16 step of the value plus an eighth of the attention tolerance is allowed
+        a, b = O_host.float(), O_dev.float()
+        bound = 2.0 ** -7 * torch.maximum(a.abs(), b.abs()) + hp.ATT_MAX_ABS / 8
+        assert bool(((a - b).abs() <= bound).all()), float((a - b).abs().max())
+    else:
+        assert torch.equal(O_host, O_dev)
     want = orc.attend(syn.bf16_bits_to_f64(Qb), hp.torch_to_f64(seq.K[0]), hp.torch_to_f64(seq.V[0]), sel, t, p,
                       heads=[0, cfg.H - 1])
     hp.check_attention(O_host[0], want, what=f"host K/V {name} t={t} l_C={l_C}", heads=[0, cfg.H - 1])
