@@ -154,7 +154,19 @@ esa_status esa_select_full_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int
  * ESA_ERR_INDEX is recorded in the device status word).  O: device [B, l_C, H, d]
  * bf16.  Query head h reads key/value head h / (H/H_G).  Query c of the chunk attends
  * every I, selected-M and L key and the keys of C at chunk offsets <= c; bf16 products,
- * fp32 softmax and accumulation. */
+ * fp32 softmax and accumulation.
+ *
+ * Ordering.  The call is ordered after everything enqueued on its stream before it, with one
+ * exception that the caller must know.  A call that is the first esa_attend* on `stream` after an
+ * esa_select* made through the same context on the same stream (the usual step: select, then
+ * attend) reads the cache rows older than the chunk (positions < n_prev[b]: the rows of I and L)
+ * while the selection kernels may still be running, and only then waits for the work ahead of it
+ * in the stream; those rows do not depend on the selection (Section 3.2: I and L are always kept).
+ * Between such a pair of calls the caller therefore enqueues nothing on the stream that writes K
+ * or V rows at positions < n_prev[b]; rows of the chunk itself (esa_append_kv), idx, n_sel and
+ * anything else may be written there.  Any other esa_attend call starts all of its reads after
+ * the preceding work of the stream.  The two orders add the same terms in another order: results
+ * agree to the rounding of bf16 (not bit for bit). */
 esa_status esa_attend(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C,
                       const void* K_cache, const void* V_cache, const int64_t* n_prev,
                       const int32_t* idx, const int32_t* n_sel, void* O);

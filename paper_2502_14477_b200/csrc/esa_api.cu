@@ -106,6 +106,12 @@ esa_status build_meta(const esa_ctx* ctx, int B, const int64_t* n_prev, int64_t 
 
 esa_status from_cuda(cudaError_t e) { return e == cudaSuccess ? ESA_OK : ESA_ERR_CUDA; }
 
+// The selection of a step has been enqueued on `st`: the attention call that follows it there may start early.
+void arm_attention(esa_ctx* ctx, cudaStream_t st) {
+    ctx->sel_armed = true;
+    ctx->sel_stream = st;
+}
+
 }  // namespace
 
 extern "C" {
@@ -177,6 +183,9 @@ esa_status esa_create(const esa_config* cfg, esa_ctx** out) {
     c->sel_ticket = reinterpret_cast<int*>(base + L.ticket);
     c->sel_slice_stride = (int)L.slice_stride;
     c->last_decode = false;
+    c->sel_armed = false;
+    c->sel_stream = nullptr;
+    c->attend_early = false;
     c->att_part = reinterpret_cast<float*>(base + L.att);
     c->att_part_elems = L.att_elems;
     c->att_count = reinterpret_cast<int*>(base + L.att_count);
@@ -319,7 +328,10 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
         e = launch_select_all(ctx, B, meta, idx_out, n_sel_out, st);
         if (e != cudaSuccess) return ESA_ERR_CUDA;
     }
-    if (!any_large) return ESA_OK;
+    if (!any_large) {
+        arm_attention(ctx, st);
+        return ESA_OK;
+    }
     // q' = f_q(q) (Eq. 5)
     RowMap zero;
     for (int b = 0; b < kMaxBatch; ++b) zero.row0[b] = 0;
@@ -355,6 +367,7 @@ esa_status esa_select_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t 
                      &pooled_ready);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
     e = launch_select(ctx, B, l_C == 1, smeta, max_lM, pooled_ready, idx_out, n_sel_out, st);
+    if (e == cudaSuccess) arm_attention(ctx, st);
     return from_cuda(e);
 }
 
@@ -379,7 +392,10 @@ esa_status esa_select_full_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int
     ctx->last_scored = any_large;
     ctx->last_q_rows = 0;
     if (any_small && launch_select_all(ctx, B, meta, idx_out, n_sel_out, st) != cudaSuccess) return ESA_ERR_CUDA;
-    if (!any_large) return ESA_OK;
+    if (!any_large) {
+        arm_attention(ctx, st);
+        return ESA_OK;
+    }
     SeqMeta smeta = meta;
     for (int b = 0; b < B; ++b)
         if (meta.m_end[b] - meta.i_end[b] <= ctx->cfg.top_k) smeta.m_end[b] = smeta.i_end[b];
@@ -387,7 +403,9 @@ esa_status esa_select_full_async(esa_ctx* ctx, int32_t B, const void* Q_cur, int
     cudaError_t e = launch_score_full(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)K_cache, smeta, max_lM,
                                       mode == ESA_SCORE_PER_HEAD, st);
     if (e != cudaSuccess) return ESA_ERR_CUDA;
-    return from_cuda(launch_select(ctx, B, false, smeta, max_lM, false, idx_out, n_sel_out, st));
+    e = launch_select(ctx, B, false, smeta, max_lM, false, idx_out, n_sel_out, st);
+    if (e == cudaSuccess) arm_attention(ctx, st);
+    return from_cuda(e);
 }
 
 esa_status esa_select_full(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_cache,
@@ -416,10 +434,15 @@ esa_status esa_attend_two_position_async(esa_ctx* ctx, int32_t B, const void* Q_
     SeqMeta meta;
     s = build_meta(ctx, B, n_prev, l_C, &meta, nullptr);
     if (s != ESA_OK) return s;
-    return from_cuda(launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)Q_far,
-                                   (const __nv_bfloat16*)K_cache, (const __nv_bfloat16*)K_far_cache,
-                                   (const __nv_bfloat16*)V_cache, meta, idx, n_sel, (__nv_bfloat16*)O,
-                                   (cudaStream_t)stream));
+    // a call that follows the selection of its step on the same stream may attend the older rows early
+    ctx->attend_early = ctx->sel_armed && ctx->sel_stream == (cudaStream_t)stream;
+    ctx->sel_armed = false;
+    cudaError_t e = launch_attend(ctx, B, l_C, (const __nv_bfloat16*)Q_cur, (const __nv_bfloat16*)Q_far,
+                                  (const __nv_bfloat16*)K_cache, (const __nv_bfloat16*)K_far_cache,
+                                  (const __nv_bfloat16*)V_cache, meta, idx, n_sel, (__nv_bfloat16*)O,
+                                  (cudaStream_t)stream);
+    ctx->attend_early = false;
+    return from_cuda(e);
 }
 
 esa_status esa_attend_two_position(esa_ctx* ctx, int32_t B, const void* Q_cur, const void* Q_far, int32_t l_C,
@@ -466,6 +489,7 @@ esa_status esa_attend_host_kv_async(esa_ctx* ctx, int32_t B, const void* Q_cur, 
     }
     if (stage_rows >= (int64_t(1) << 31)) return ESA_ERR_CAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
+    ctx->sel_armed = false;       // (the staged list is written by the gather kernel just ahead: never attended early)
     if (launch_gather_kv(ctx, B, l_C, K_host, V_host, meta, idx, n_sel, K_stage, V_stage, stage_rows, st) != cudaSuccess)
         return ESA_ERR_CUDA;
     // The staged rows are the attended list itself: the attention kernels run on the same partition with the

@@ -39,6 +39,7 @@ struct AttendParams {
     int* unit_count;          // arrival counters per (sequence, key/value head) for the in-kernel merge of the decode kernel
     int* status;              // device status word (may be null: the entry point without a context)
     int staged;               // the caches hold the attended list itself: row j = list entry j
+    int early;                // the older rows of L may be attended ahead of the wait for the preceding kernel
     int64_t max_tokens;
     int l_C, H, HG, G, top_k;
     int nsplit;
@@ -404,7 +405,7 @@ attend_decode_kernel(AttendParams p) {
     // still at work on a handful of SMs, and its share of the rest of the list after it (phase 1, list positions).
     // (Not with two position encodings, nor when the caches hold the staged list: phase 1 alone does everything.)
     const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
-    const bool early = !TWO && !p.staged;
+    const bool early = !TWO && p.early;
     const int u_pre = early ? ((t - m_end) / DEC_ROWS) * DEC_ROWS : 0;     // rows of L done in phase 0: whole iterations
     const int itA_all = u_pre / DEC_ROWS;
     const int perA = (itA_all + p.nsplit - 1) / p.nsplit;
@@ -789,6 +790,7 @@ cudaError_t launch_attend(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* Q, 
     p.V = V; p.O = O; p.idx = idx; p.n_sel = n_sel; p.part = ctx->att_part; p.unit_count = nullptr;
     p.status = ctx->status;
     p.staged = staged ? 1 : 0;
+    p.early = ctx->attend_early && !two && !staged ? 1 : 0;
     p.max_tokens = cache_rows > 0 ? cache_rows : ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;
@@ -915,7 +917,7 @@ extern "C" esa_status esa_attend_noalloc(const esa_config* cfg, int32_t B, const
     AttendParams p;
     p.Q = (const __nv_bfloat16*)Q_cur; p.K = (const __nv_bfloat16*)K_cache; p.V = (const __nv_bfloat16*)V_cache;
     p.Qg = p.Q; p.Kg = p.K;
-    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr; p.staged = 0;
+    p.O = (__nv_bfloat16*)O; p.idx = idx; p.n_sel = n_sel; p.part = dev.part; p.unit_count = nullptr; p.status = nullptr; p.staged = 0; p.early = 0;
     p.max_tokens = cfg->max_tokens; p.l_C = l_C; p.H = cfg->n_q_heads; p.HG = cfg->n_kv_heads; p.G = G;
     p.top_k = cfg->top_k; p.nsplit = 1;
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)D);

@@ -85,6 +85,7 @@ struct TcAttendParams {
     int* unit_count;    // arrivals per (sequence, key/value head, row tile); returns to 0 after each launch
     int q_tma;          // Q tiles arrive by TMA (one arrival) instead of cp.async (one per producer thread)
     int staged;         // the caches hold the attended list itself: row j = list entry j
+    int early;          // the rows of I and L are attended ahead of the wait for the preceding kernel (never with staged or two)
     int two;            // two-position attention: splits [0, nsplit/2) take I and M_k with (Qg, Kg), the rest L and C with (Q, K)
     float scale_log2;
     SeqMeta meta;
@@ -250,31 +251,55 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     // columns: S of Q tile q at q * 128 (half u at + u * 64); O of Q tile q at 256 + q * D
-    // everything read from global memory comes after the preceding kernel (the selection) is complete
-    pdl_wait();
-    pdl_launch_dependents();
+    // The rows of I and L are older than the chunk and depend on nothing the preceding kernels of the step write (the
+    // selection least of all).  With `p.early` the attended set is taken as two lists: the early one, I then L, whose
+    // tiles every CTA shares out and attends BEFORE its wait for the preceding kernel (the selection kernel is then
+    // still at work on a handful of SMs), and the late one, the selected entries then C, attended after the wait.
+    // Otherwise (two position encodings, caches that hold the staged list, or a call that does not follow the
+    // selection of its step) there is one list, I, M_k, L, C, and all of it comes after the wait.
+    // A list is described by four numbers: entry j is cache row j below `ie`, idx[j - ie] below `ng`, cache row
+    // me + (j - ng) from there on, and nothing from `row_lim` on.
+    struct KeyList { int ie, ng, me, row_lim; };
     const int t = p.meta.t[b], i_end = p.meta.i_end[b], m_end = p.meta.m_end[b];
-    int n_sel = p.n_sel[b];
-    n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
-    const int n_glob = i_end + n_sel;
-    const int n_att = n_glob + (t - m_end) + p.l_C;
-    const int c_first = n_att - p.l_C;
-
     const int r_last = min(R, row0 + TC_ROWS) - 1;
-    const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
-    // The part of the key list this CTA's group of splits covers: all of it, or (two-position attention)
-    // the entries of I and M_k for the first half of the splits and those of L and C for the second.
-    const int grp = p.two ? p.nsplit / 2 : p.nsplit;       // splits that share a part
-    const bool far = p.two && split < grp;                 // this CTA works with (Qg, Kg)
-    const int part_lo = (p.two && !far) ? n_glob : 0;
-    const int part_hi = far ? n_glob : j_end;
-    const int s_in = (p.two && !far) ? split - grp : split;
-    const int n_tiles_all = max(0, (part_hi - part_lo + TC_BN - 1) / TC_BN);
-    const int per = (n_tiles_all + grp - 1) / grp;
-    const int tile_begin = s_in * per;
-    const int tile_end = min(n_tiles_all, tile_begin + per);
-    const int n_tiles = max(0, tile_end - tile_begin);
-    auto tile_key0 = [&](int T) { return part_lo + (tile_begin + T) * TC_BN; };   // first list position of the CTA's T-th tile
+    const int e_len = p.early ? i_end + (t - m_end) : 0;                 // entries of the early list
+    const int early_all = (e_len + TC_BN - 1) / TC_BN;
+    const int early_per = (early_all + p.nsplit - 1) / p.nsplit;
+    const int early_begin = min(early_all, split * early_per);
+    const int n_early = min(early_all, early_begin + early_per) - early_begin;      // this CTA's early tiles
+    const KeyList list_early = {i_end, i_end, m_end, e_len};
+    // set after the wait: the late (or only) list, this CTA's part of it, and the tile count of both phases
+    KeyList list_late = {0, 0, 0, 0};
+    int c_first = 0, part_lo = 0, part_hi = 0, tile_begin = 0, n_tiles = 0;
+    bool far = false, planned = false;
+    auto plan = [&]() {
+        pdl_wait();
+        pdl_launch_dependents();
+        int n_sel = p.n_sel[b];
+        n_sel = max(0, min(n_sel, min(p.top_k, m_end - i_end)));
+        if (p.early) list_late = {0, n_sel, t, n_sel + p.l_C};
+        else list_late = {i_end, i_end + n_sel, m_end, i_end + n_sel + (t - m_end) + p.l_C};
+        c_first = list_late.row_lim - p.l_C;                  // entry of the chunk's first token
+        const int j_end = c_first + r_last / G + 1;           // keys visible to the last row of the CTA
+        // The part of the key list this CTA's group of splits covers: all of it, or (two-position attention)
+        // the entries of I and M_k for the first half of the splits and those of L and C for the second.
+        const int grp = p.two ? p.nsplit / 2 : p.nsplit;       // splits that share a part
+        far = p.two && split < grp;                            // this CTA works with (Qg, Kg)
+        part_lo = (p.two && !far) ? list_late.ng : 0;
+        part_hi = far ? list_late.ng : j_end;
+        if (far) list_late.row_lim = part_hi;
+        // (with an early list the shares run the other way round: the split with the short early share comes first)
+        const int s_in = (p.two && !far) ? split - grp : (p.early ? grp - 1 - split : split);
+        const int late_all = max(0, (part_hi - part_lo + TC_BN - 1) / TC_BN);
+        const int per = (late_all + grp - 1) / grp;
+        tile_begin = min(late_all, s_in * per);
+        n_tiles = n_early + min(late_all, tile_begin + per) - tile_begin;
+        planned = true;
+    };
+    if (n_early == 0) plan();
+    // Every role takes its tiles in two phases, the early ones and, after `plan`, the late ones; tile j of the CTA
+    // starts at entry key_first + (j - j_first) * TC_BN of the phase's list.
+    const bool has_work = n_early > 0 || n_tiles > 0;
 
     if (warp_u < TC_SOFTMAX_WARPS) reg_alloc<TC_REGS_SOFTMAX>();
     else reg_dealloc<TC_REGS_OTHER>();
@@ -286,15 +311,21 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         const int row = row0 + qt * 128 + lane_base + lane;
         const uint32_t tS = tmem_addr(tmem, lane_base, qt * 128);
         const uint32_t tO = tmem_addr(tmem, lane_base, 256 + qt * D);
-        // first invisible list position of this row, and the smallest such limit of the Q tile
-        const int lim = min(part_hi, c_first + min(row / G, p.l_C - 1) + 1);
-        const int lim_min = min(part_hi, c_first + min((row0 + qt * 128) / G, p.l_C - 1) + 1);
         const float sl2 = p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
 
-        for (int j = 0; j < 2 * n_tiles; ++j) {             // j counts halves: tile j >> 1, half j & 1
+#pragma unroll 1
+        for (int phase = 0; phase < 2; ++phase) {
+        if (phase == 1 && !planned) plan();
+        const int j_first = phase == 0 ? 0 : 2 * n_early, j_last = phase == 0 ? 2 * n_early : 2 * n_tiles;
+        const int key_first = phase == 0 ? early_begin * TC_BN : part_lo + tile_begin * TC_BN;
+        // first invisible entry of this row, and the smallest such limit of the Q tile (every row sees all of the
+        // early list)
+        const int lim = phase == 0 ? e_len : min(part_hi, c_first + min(row / G, p.l_C - 1) + 1);
+        const int lim_min = phase == 0 ? e_len : min(part_hi, c_first + min((row0 + qt * 128) / G, p.l_C - 1) + 1);
+        for (int j = j_first; j < j_last; ++j) {            // j counts halves: tile j >> 1, half j & 1
             const int T = j >> 1, u = j & 1;
-            const int key0 = tile_key0(T) + u * TC_HALF;
+            const int key0 = key_first + (j - j_first) * TC_HALF;
             if (u == 0) {
                 mbar_wait(bar(BAR_S_READY + qt), T & 1, wc);
                 tc_fence_after_sync();
@@ -376,6 +407,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(bar(BAR_P_READY + qt * 2 + u));
+        }
         }
 
         // ---- epilogue: O / l  (or the unnormalised partial for the split merge)
@@ -686,7 +718,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
     } else if (warp_u < TC_MMA_WARP) {
         // ------------------------------------------------------------ producers: Q, then K/V tiles
         const int ptid = tid - TC_SOFTMAX_WARPS * 32;      // 0..127
-        if (n_tiles > 0 && p.q_tma) {
+        if (has_work && p.q_tma) {
             // two boxes per 64-column block: rows (query, head-in-group) of one key/value head
             if (ptid == 0) {
                 mbar_arrive_expect_tx(bar(BAR_Q_FULL), 2 * Q_TILE_BYTES);
@@ -698,7 +730,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                         tma_load_3d(smem_u32(sQ + qt * Q_TILE_BYTES + blk * Q_BLK_BYTES), qm, blk * 64, kvh * G,
                                     b * p.l_C + (row0 + qt * 128) / G, bar(BAR_Q_FULL));
             }
-        } else if (n_tiles > 0) {
+        } else if (has_work) {
             // group sizes that do not divide 128: 16-byte copies, row by row
             const int chunk = ptid % CH, rsub = ptid / CH, cin = chunk & 7;
             constexpr int RSTEP = TC_PRODUCERS / CH;
@@ -722,7 +754,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         constexpr int NPASS = TC_BN / RPP;                 // 4
         constexpr int CPT = CH / TPR;                      // chunks per thread and row: 4 (D = 128) or 2
         const int q4 = ptid % TPR, rfirst = ptid / TPR;
-        const __nv_bfloat16* Kb = (far ? p.Kg : p.K) + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
+        const __nv_bfloat16* Kb0 = p.K + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
+        const __nv_bfloat16* Kb1 = p.Kg + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const __nv_bfloat16* Vb = p.V + ((int64_t)b * p.max_tokens * p.HG + kvh) * D + q4 * 8;
         const int32_t* idx = p.idx + (int64_t)b * p.top_k;
         const int64_t tok_stride = (int64_t)p.HG * D;
@@ -733,24 +766,29 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             const int r = rfirst + it * RPP;
             row_off[it] = (uint32_t)(r * 128) | (uint32_t)((r & 7) << 4);      // XOR with (c & 7) << 4 gives the swizzled chunk
         }
-        const int row_lim = far ? part_hi : n_att;          // list positions of this CTA's part end here
         int bad_idx = 0;
-        for (int j = 0; j < n_tiles; ++j) {
+#pragma unroll 1
+        for (int phase = 0; phase < 2; ++phase) {
+        if (phase == 1 && !planned) plan();
+        const KeyList kl = phase == 0 ? list_early : list_late;
+        const int j_first = phase == 0 ? 0 : n_early, j_last = phase == 0 ? n_early : n_tiles;
+        const int key_first = phase == 0 ? early_begin * TC_BN : part_lo + tile_begin * TC_BN;
+        for (int j = j_first; j < j_last; ++j) {
             const int s = j % STAGES;
             const uint32_t ph = ((j / STAGES) & 1) ^ 1;
-            const int key0 = tile_key0(j);
+            const int key0 = key_first + (j - j_first) * TC_BN;
             int pos[NPASS];
             uint32_t from_idx = 0;                      // rows whose position was read from the selection
 #pragma unroll
             for (int it = 0; it < NPASS; ++it) {
                 const int jj = key0 + rfirst + it * RPP;
                 int q = -1;
-                if (jj >= row_lim) q = -1;
-                else if (p.staged || jj < i_end) q = jj;
-                else if (jj < n_glob) {
-                    q = __ldg(idx + (jj - i_end));
+                if (jj >= kl.row_lim) q = -1;
+                else if (p.staged || jj < kl.ie) q = jj;
+                else if (jj < kl.ng) {
+                    q = __ldg(idx + (jj - kl.ie));
                     from_idx |= 1u << it;
-                } else q = m_end + (jj - n_glob);
+                } else q = kl.me + (jj - kl.ng);
                 pos[it] = q;
             }
             mbar_wait(bar(BAR_K_EMPTY + s), ph, wc);
@@ -761,7 +799,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 if ((from_idx >> it) & 1u) pos[it] = clamp_selected(pos[it], i_end, m_end, bad_idx);
 #pragma unroll
             for (int it = 0; it < NPASS; ++it) {
-                const __nv_bfloat16* src = Kb + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
+                const __nv_bfloat16* src = (far ? Kb1 : Kb0) + (pos[it] < 0 ? 0 : pos[it]) * tok_stride;
                 const int nbytes = pos[it] < 0 ? 0 : 16;
                 uint8_t* tile = sK + s * KV_TILE_BYTES;
 #pragma unroll
@@ -785,9 +823,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
             }
             cp_async_arrive_noinc(bar(BAR_V_FULL + s));
         }
+        }
         if (bad_idx) atomicExch(p.status, kStatusBadIndex);
         cp_async_wait<0>();
-    } else if (warp_u == TC_MMA_WARP && n_tiles > 0) {
+    } else if (warp_u == TC_MMA_WARP && has_work) {
         // ------------------------------------------------------------ MMA issue: one converged warp, lane 0 leads.
         // The fixed order (Q tile 0's products of a tile, then Q tile 1's) keeps the two Q tiles half a period
         // apart: S of Q tile 1 always becomes ready one block of products after S of Q tile 0, so each softmax
@@ -823,10 +862,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         issue_qk(1, 0);
         umma_commit(bar(BAR_S_READY + 1), lead);
         umma_commit(bar(BAR_K_EMPTY + 0), lead);
-        for (int T = 0; T < n_tiles; ++T) {
+        for (int T = 0; !planned || T < n_tiles; ++T) {
             const int s = T % STAGES;
             const int Tn = T + 1, sn = Tn % STAGES;
-            const bool more = Tn < n_tiles;
+            // Whether a tile follows the last early one is known only after the wait for the preceding kernel: that
+            // round ends like a last one, and the products of the first late tile are issued once the wait is over.
+            const bool defer = !planned && Tn >= n_early;
+            const bool more = !defer && (!planned || Tn < n_tiles);
             mbar_wait(bar(BAR_V_FULL + s), (T / STAGES) & 1, wc);
             fence_async_smem();
 #pragma unroll
@@ -843,12 +885,27 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 tc_fence_after_sync();
                 issue_pv(qt, s, 1, 1);
                 umma_commit(bar(BAR_PV_DONE + qt), lead);
-                if (!more) umma_commit(bar(BAR_O_READY + qt), lead);
+                if (!more && !defer) umma_commit(bar(BAR_O_READY + qt), lead);
                 if (qt == 1) umma_commit(bar(BAR_V_EMPTY + s), lead);
                 if (more) {
                     issue_qk(qt, sn);         // overwrites S and P of this tile after the P V products above, in issue order
                     umma_commit(bar(BAR_S_READY + qt), lead);
                     if (qt == 1) umma_commit(bar(BAR_K_EMPTY + sn), lead);
+                }
+            }
+            if (defer) {
+                plan();
+                if (Tn < n_tiles) {
+                    mbar_wait(bar(BAR_K_FULL + sn), (Tn / STAGES) & 1, wc);
+                    fence_async_smem();
+                    issue_qk(0, sn);
+                    umma_commit(bar(BAR_S_READY + 0), lead);
+                    issue_qk(1, sn);
+                    umma_commit(bar(BAR_S_READY + 1), lead);
+                    umma_commit(bar(BAR_K_EMPTY + sn), lead);
+                } else {
+                    umma_commit(bar(BAR_O_READY + 0), lead);
+                    umma_commit(bar(BAR_O_READY + 1), lead);
                 }
             }
         }
@@ -965,6 +1022,7 @@ cudaError_t launch_attend_tc(esa_ctx* ctx, int B, int l_C, const __nv_bfloat16* 
     p.unit_count = ctx->att_count;
     p.staged = staged ? 1 : 0;
     p.two = two ? 1 : 0;
+    p.early = ctx->attend_early && !two && !staged ? 1 : 0;
     p.max_tokens = cache_rows > 0 ? cache_rows : ctx->cfg.max_tokens; p.l_C = l_C; p.H = ctx->H; p.HG = ctx->HG; p.G = ctx->G;
     p.top_k = ctx->cfg.top_k; p.nsplit = 1;
     p.scale_log2 = ctx->scale * 1.4426950408889634f;

@@ -82,6 +82,13 @@ struct esa_ctx {
     int* sel_ticket;     // [max_batch] arrival tickets of the selection kernel; 0 between launches
     int sel_slice_stride;
     bool last_decode;    // the last selection ran with l_C = 1 (pkey holds raw pooled scores)
+    // The attention kernels may read cache rows older than the chunk ahead of their wait for the preceding kernel
+    // only when the work ahead of them in the stream is known not to write such rows: a selection enqueued through
+    // this context arms the next attention call on the same stream (the caller's side of it: nothing enqueued
+    // between the two calls writes cache rows older than the chunk).
+    bool sel_armed;
+    cudaStream_t sel_stream;
+    bool attend_early;   // set around the launch of an armed attention call
     float* att_part;     // split-KV partial outputs + (m, l)
     size_t att_part_elems;
     int* att_count;      // arrival counters of the split prefill attention, one per (sequence, kv head, row tile); 0 between launches
