@@ -865,10 +865,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         for (int T = 0; !planned || T < n_tiles; ++T) {
             const int s = T % STAGES;
             const int Tn = T + 1, sn = Tn % STAGES;
-            // Whether a tile follows the last early one is known only after the wait for the preceding kernel: that
-            // round ends like a last one, and the products of the first late tile are issued once the wait is over.
-            const bool defer = !planned && Tn >= n_early;
-            const bool more = !defer && (!planned || Tn < n_tiles);
+            // Whether a tile follows the last early one is known only after the wait for the preceding kernel: this
+            // warp takes the wait at the start of that tile's round (by then the preceding kernel has finished, unless
+            // the early list is short), so that the round can issue the first late tile's products like any other.
+            if (!planned && Tn >= n_early) plan();
+            const bool more = !planned || Tn < n_tiles;
             mbar_wait(bar(BAR_V_FULL + s), (T / STAGES) & 1, wc);
             fence_async_smem();
 #pragma unroll
@@ -885,27 +886,12 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
                 tc_fence_after_sync();
                 issue_pv(qt, s, 1, 1);
                 umma_commit(bar(BAR_PV_DONE + qt), lead);
-                if (!more && !defer) umma_commit(bar(BAR_O_READY + qt), lead);
+                if (!more) umma_commit(bar(BAR_O_READY + qt), lead);
                 if (qt == 1) umma_commit(bar(BAR_V_EMPTY + s), lead);
                 if (more) {
                     issue_qk(qt, sn);         // overwrites S and P of this tile after the P V products above, in issue order
                     umma_commit(bar(BAR_S_READY + qt), lead);
                     if (qt == 1) umma_commit(bar(BAR_K_EMPTY + sn), lead);
-                }
-            }
-            if (defer) {
-                plan();
-                if (Tn < n_tiles) {
-                    mbar_wait(bar(BAR_K_FULL + sn), (Tn / STAGES) & 1, wc);
-                    fence_async_smem();
-                    issue_qk(0, sn);
-                    umma_commit(bar(BAR_S_READY + 0), lead);
-                    issue_qk(1, sn);
-                    umma_commit(bar(BAR_S_READY + 1), lead);
-                    umma_commit(bar(BAR_K_EMPTY + sn), lead);
-                } else {
-                    umma_commit(bar(BAR_O_READY + 0), lead);
-                    umma_commit(bar(BAR_O_READY + 1), lead);
                 }
             }
         }
