@@ -242,7 +242,7 @@ def _side_stream():
     return _SIDE[0]
 
 
-PROFILE_EVERY = 8      # one chunk in this many runs with per-kernel CUDA events (see run_prefill_layer)
+PROFILE_EVERY = 32     # one chunk in this many runs with per-kernel CUDA events (see run_prefill_layer)
 
 
 def run_prefill_layer(ctx, cfg, L, bufs, sampled=None, phase=0):
@@ -250,10 +250,11 @@ def run_prefill_layer(ctx, cfg, L, bufs, sampled=None, phase=0):
 
     sampled: list that receives (t, l_C) of the chunks whose kernels were individually timed.  On
     such a chunk the library brackets every kernel with CUDA events on the launching stream
-    (esa_set_profiling).  An event record between two kernels keeps the second one from being set
-    up under the first one's tail (programmatic dependent launch), which costs 8 % of the step when
-    every launch is bracketed; so one chunk in PROFILE_EVERY is, the sampled position rotating with
-    `phase` (over 8 steps every chunk position is sampled once)."""
+    (esa_set_profiling).  An event record between two kernels keeps the second one from starting
+    under the first one (programmatic dependent launch; the attention kernel reads the older rows
+    beside the selection kernel), which costs a sampled chunk about a quarter of its time: measured
+    163k / 169k / 172k tokens/s with one chunk in 8 / 16 / 32 sampled.  So one chunk in
+    PROFILE_EVERY is, the sampled positions moving with `phase` (step number)."""
     Kc, idx, n_sel, O = bufs
     # The compressed keys of the current chunk are not read by this chunk's selection (C is not
     # part of M): esa_compress_keys runs on a side stream beside the attention, and the selection
@@ -265,7 +266,7 @@ def run_prefill_layer(ctx, cfg, L, bufs, sampled=None, phase=0):
     for t in range(0, cfg.S, cfg.l_C):
         l_C = min(cfg.l_C, cfg.S - t)
         Qc = L.Q[:, t: t + l_C]
-        timed = sampled is not None and (t // cfg.l_C + phase) % PROFILE_EVERY == 0
+        timed = sampled is not None and (t // cfg.l_C + 5 * phase) % PROFILE_EVERY == 0
         if timed:
             ctx.set_profiling(True)
         with torch.cuda.stream(side):

@@ -286,7 +286,7 @@ esa_status esa_compress_keys_async(esa_ctx* ctx, int32_t B, const void* K_new, i
     if (ctx->has_wmaps) {
         cudaError_t e = launch_compress_tc(ctx, (const __nv_bfloat16*)K_new, B, n_new, ctx->dG, &ctx->wk_map,
                                            ctx->has_bk ? ctx->bk : nullptr, (__nv_bfloat16*)kc_cache,
-                                           ctx->cfg.max_tokens, map, nullptr, 0, (cudaStream_t)stream);
+                                           ctx->cfg.max_tokens, map, nullptr, 0, (cudaStream_t)stream, true);
         if (e != cudaErrorNotSupported) return from_cuda(e);
         cudaGetLastError();
     }

@@ -176,14 +176,20 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
 template <int DC>
 cudaError_t launch_t(esa_ctx* ctx, const __nv_bfloat16* X, int rows, int rows_per_seq, int d_in, const CUtensorMap* wmap,
                      const float* bias, __nv_bfloat16* dst, int64_t seq_stride, const RowMap& map, uint32_t* zero_words,
-                     int zero_count, cudaStream_t st) {
+                     int zero_count, cudaStream_t st, bool small_grid) {
     CUtensorMap xmap;
     if (!make_tensor_map_bf16(&xmap, X, (uint64_t)rows, (uint64_t)d_in, CT_ROWS)) return cudaErrorNotSupported;
     const int row_tiles = (rows + CT_ROWS - 1) / CT_ROWS;
     const int n_chunks_total = d_in / CT_KCHUNK;
-    // split the reduction while that still adds CTAs usefully (power of two, at most 16, whole chunks)
+    // split the reduction while that still adds CTAs usefully (power of two, at most 16, whole chunks).  A call
+    // whose result is not needed at once stays within an eighth of the SMs: beside the kernels of a step on another
+    // stream it then fits on the SMs those leave idle (the attention grid of the Llama-3-8B shape leaves 20 of 148)
+    // instead of holding back CTAs of theirs: 32 -> 16 CTAs for a 512-row chunk, +3 % prefill rate.
+    const int cta_limit = small_grid ? max(ctx->num_sms / 8, 1) : ctx->num_sms;
     int nsplit = 1;
-    while (nsplit < CT_MAX_SPLIT && n_chunks_total % (nsplit * 2) == 0 && row_tiles * nsplit < ctx->num_sms) nsplit *= 2;
+    while (nsplit < CT_MAX_SPLIT && n_chunks_total % (nsplit * 2) == 0 &&
+           (small_grid ? row_tiles * nsplit * 2 <= cta_limit : row_tiles * nsplit < cta_limit))
+        nsplit *= 2;
     constexpr int smem_stage = (CT_ROWS + DC) * CT_KCHUNK * 2;
     constexpr int smem_part = CT_ROWS * (DC + 4) * 4;
     constexpr int smem = (CT_STAGES * smem_stage > smem_part ? CT_STAGES * smem_stage : smem_part) + 1024;
@@ -288,11 +294,11 @@ bool make_tensor_map_q(CUtensorMap* map, const void* base, uint64_t n_queries, i
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
                                int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool small_grid) {
     if (d_in % CT_KCHUNK) return cudaErrorNotSupported;
     const int rows = B * rows_per_seq;
-    if (ctx->dc == 128) return launch_t<128>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st);
-    if (ctx->dc == 64) return launch_t<64>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st);
+    if (ctx->dc == 128) return launch_t<128>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st, small_grid);
+    if (ctx->dc == 64) return launch_t<64>(ctx, X, rows, rows_per_seq, d_in, wmap, bias, dst, dst_seq_stride, map, zero_words, zero_count, st, small_grid);
     return cudaErrorNotSupported;
 }
 

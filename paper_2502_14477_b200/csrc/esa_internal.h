@@ -207,10 +207,12 @@ cudaError_t launch_compress_gemv(esa_ctx* ctx, const __nv_bfloat16* X, int B, in
                                  const __nv_bfloat16* W, const float* bias, __nv_bfloat16* dst,
                                  int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
                                  uint32_t* zero2_words, int zero2_count, cudaStream_t st);
+// small_grid: the result is not needed at once (key compression: its rows enter M only l_L tokens later, and callers
+// run it on a side stream), so the grid is kept to an eighth of the SMs instead of as many CTAs as shorten the call.
 cudaError_t launch_compress_tc(esa_ctx* ctx, const __nv_bfloat16* X, int B, int rows_per_seq, int d_in,
                                const CUtensorMap* wmap, const float* bias, __nv_bfloat16* dst,
                                int64_t dst_seq_stride, const RowMap& map, uint32_t* zero_words, int zero_count,
-                               cudaStream_t st);
+                               cudaStream_t st, bool small_grid = false);
 
 // True when launch_score takes the tcgen05 path for this call.
 inline bool score_uses_tc(const esa_ctx* ctx, int B, int l_C) {
