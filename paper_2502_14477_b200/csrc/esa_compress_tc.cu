@@ -148,19 +148,17 @@ compress_tc_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_consta
         const int lr = split * band + i / PER_ROW, c4 = (i % PER_ROW) * 4;
         const int row = row0 + lr;
         if (row >= p.rows) continue;
-        // remote reads four at a time (their latencies overlap); the sum order stays split order
+        // all remote reads of an element in flight together (a read from another CTA's shared memory takes most of
+        // a microsecond); the sum order stays split order
+        float4 v[CT_MAX_SPLIT];
+#pragma unroll
+        for (int j = 0; j < CT_MAX_SPLIT; ++j)
+            v[j] = j < nsplit ? *reinterpret_cast<const float4*>(cluster.map_shared_rank(sPart, j) + lr * PSTRIDE + c4)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp0 = 0; sp0 < nsplit; sp0 += 4) {
-            float4 v[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                v[j] = sp0 + j < nsplit
-                           ? *reinterpret_cast<const float4*>(cluster.map_shared_rank(sPart, sp0 + j) + lr * PSTRIDE + c4)
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                s.x += v[j].x; s.y += v[j].y; s.z += v[j].z; s.w += v[j].w;
-            }
+        for (int j = 0; j < CT_MAX_SPLIT; ++j) {
+            s.x += v[j].x; s.y += v[j].y; s.z += v[j].z; s.w += v[j].w;
         }
         if (p.bias) {
             s.x += p.bias[c4]; s.y += p.bias[c4 + 1]; s.z += p.bias[c4 + 2]; s.w += p.bias[c4 + 3];
