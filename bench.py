@@ -40,8 +40,8 @@ import esa_synth as syn
 N_LAYERS_STACK = 32
 # dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised in
 # profiles/dram_bytes_per_kernel.txt (same kernels, same launch shapes as the timed workloads).
-ATTEND_TC_DRAM_BYTES = 32090880 + 0
-DECODE_STEP_DRAM_BYTES = (205829632 + 55296) + 39168 + 300032 + 1133568 + (264881408 + 542976) + 4354048
+ATTEND_TC_DRAM_BYTES = 32086272 + 0
+DECODE_STEP_DRAM_BYTES = (205831680 + 368128) + 39168 + 300032 + 1133312 + (264881152 + 138752) + 4355072
 
 
 # ----------------------------------------------------------------------------

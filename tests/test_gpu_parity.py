@@ -607,6 +607,16 @@ def test_attention_that_follows_its_selection_attends_the_older_rows_early(name,
     O_plain = torch.full_like(Q, float("nan"))
     ctx.attend(Q, seq.K, seq.V, [t], seq.idx, seq.n_sel, O_plain, sync=True)
     assert ctx.last_device_status() == 0
+    # a selection enqueued on another stream arms nothing: the attention call takes the list in order after its wait
+    other = torch.cuda.Stream()
+    idx2, n_sel2 = torch.zeros_like(seq.idx), torch.zeros_like(seq.n_sel)
+    other.wait_stream(torch.cuda.current_stream())
+    ctx.select(Q, seq.Kc, [t], idx2, n_sel2, stream=other)
+    other.synchronize()
+    assert torch.equal(idx2, seq.idx) and torch.equal(n_sel2, seq.n_sel)
+    O_other = torch.full_like(Q, float("nan"))
+    ctx.attend(Q, seq.K, seq.V, [t], idx2, n_sel2, O_other, sync=True)
+    assert torch.equal(O_other, O_plain)
     a, b = O_early.float(), O_plain.float()
     v_max = float(seq.V[0, :n].float().abs().max())
     bound = 2.0 ** -8 * v_max + 2.0 ** -8 * torch.maximum(a.abs(), b.abs())
