@@ -34,6 +34,12 @@
 //     halves of their partial (O, m, l) through distributed shared memory (PAIR, below); otherwise the partials
 //     go to the context's scratch through coalesced stores, and the CTA that finishes a unit last merges
 //     them with its own accumulator (an arrival counter per unit decides; nobody waits).
+//   * A call that follows the selection of its step (p.early) takes the attended set as two lists: I then L,
+//     whose rows are older than the chunk and do not depend on the selection, before the kernel's wait for the
+//     preceding kernel, and M_k then C after it.  Every role runs the two phases in turn; the selection kernel
+//     (a handful of busy SMs) runs beside the first.  The issuing warp takes the wait at the start of the last
+//     early tile's round; one issuing warp it stays (two, sharing the k-steps of every product, were slower
+//     whether they alternated strictly or ran freely, and the free-running pair gave up the fixed order of sums).
 //   * Two-position attention (Section 3.2) is a split by construction: the first half of the splits
 //     covers the list entries of I and M_k with the second encoding (Qg, Kg), the other half covers
 //     L and C with (Q, K), so a CTA holds one pair of Q tiles whichever part it works on, and the
