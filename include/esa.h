@@ -94,7 +94,8 @@ esa_status esa_destroy(esa_ctx* ctx);
  * Wq [d_c, H*d], Wk [d_c, H_G*d] (row-major; a key compressor defined on H repeated
  * heads folds to this shape by summing each group's columns), bq/bk [d_c] or NULL for
  * no bias.  Weights are rounded once to bf16 (round-to-nearest-even) and copied to
- * the device; biases stay fp32.  Synchronous. */
+ * the device; biases stay fp32.  Synchronous copies on the default stream: work of this
+ * context that is still in flight on a non-blocking stream must be waited for first. */
 esa_status esa_set_compressors(esa_ctx* ctx, const float* Wq, const float* bq,
                                const float* Wk, const float* bk);
 
@@ -205,8 +206,10 @@ esa_status esa_attend_two_position_async(esa_ctx* ctx, int32_t B, const void* Q_
  *                    l_I + top_k + l_L + l_C: the rows of I, M_k, L and C are copied there in
  *                    list order by one gather kernel (16-byte reads across PCIe), and the
  *                    attention kernels run on the staged rows.
- * Everything else is as for esa_attend; the result is bit-identical to esa_attend on
- * device-resident copies of the same caches.  ESA_ERR_CAPACITY if stage_rows is too small. */
+ * Everything else is as for esa_attend; the result is bit-identical to an esa_attend on
+ * device-resident copies of the same caches that does not follow a selection (the staged rows
+ * are written by the gather kernel just ahead, so this call never reads rows early: see
+ * "Ordering" above).  ESA_ERR_CAPACITY if stage_rows is too small. */
 esa_status esa_attend_host_kv(esa_ctx* ctx, int32_t B, const void* Q_cur, int32_t l_C, const void* K_host,
                               const void* V_host, const int64_t* n_prev, const int32_t* idx, const int32_t* n_sel,
                               void* K_stage, void* V_stage, int64_t stage_rows, void* O);
