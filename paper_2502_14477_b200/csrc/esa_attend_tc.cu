@@ -297,9 +297,18 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant
         // (with an early list the shares run the other way round: the split with the short early share comes first)
         const int s_in = (p.two && !far) ? split - grp : (p.early ? grp - 1 - split : split);
         const int late_all = max(0, (part_hi - part_lo + TC_BN - 1) / TC_BN);
-        const int per = (late_all + grp - 1) / grp;
-        tile_begin = min(late_all, s_in * per);
-        n_tiles = n_early + min(late_all, tile_begin + per) - tile_begin;
+        if (p.early && grp == 2 && late_all >= 2) {
+            // Two splits: the late list is cut where the first split's early and late tiles together make half of
+            // all tiles (rounded up).  The second split, which holds the masked tiles of C (the dearer ones), is then
+            // never the one with a tile more.
+            const int cut = min(late_all, max(0, ((early_all + late_all + 1) >> 1) - min(early_all, early_per)));
+            tile_begin = split == 0 ? 0 : cut;
+            n_tiles = n_early + (split == 0 ? cut : late_all - cut);
+        } else {
+            const int per = (late_all + grp - 1) / grp;
+            tile_begin = min(late_all, s_in * per);
+            n_tiles = n_early + min(late_all, tile_begin + per) - tile_begin;
+        }
         planned = true;
     };
     if (n_early == 0) plan();
