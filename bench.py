@@ -40,8 +40,8 @@ import esa_synth as syn
 N_LAYERS_STACK = 32
 # dram__bytes_read.sum + dram__bytes_write.sum from the ncu captures summarised in
 # profiles/dram_bytes_per_kernel.txt (same kernels, same launch shapes as the timed workloads).
-ATTEND_TC_DRAM_BYTES = 32086272 + 0
-DECODE_STEP_DRAM_BYTES = (205831680 + 368128) + 39168 + 300032 + 1133312 + (264881152 + 138752) + 4355072
+ATTEND_TC_DRAM_BYTES = 32087552 + 1280
+DECODE_STEP_DRAM_BYTES = (205836544 + 79360) + 39168 + 300288 + 1133312 + (264913408 + 626688) + 4355328
 
 
 # ----------------------------------------------------------------------------
