@@ -732,7 +732,10 @@ def run_esa(args, cfg):
                                "sampled during the run decide which applies: at the maximum SM clock, the burst one)",
                 "share_of_step": att_ms * (args.steps * n_chunks / max(1, len(sampled))) / ms_total,
                 "launches": att["launches"],
-                "sampling": "CUDA events around every kernel of 1 chunk in %d, position rotating over the steps" % PROFILE_EVERY}
+                "sampling": "CUDA events around every kernel of 1 chunk in %d, positions moving with the step; an "
+                            "event-bracketed launch runs alone, so the kernel's early phase (rows of I and L, normally "
+                            "beside the selection kernel) counts in full and share_of_step overstates its part of a "
+                            "pipelined step" % PROFILE_EVERY}
 
     # host time to enqueue a chunk (three library calls + the side-stream bookkeeping), GPU queue empty at the start
     torch.cuda.synchronize()
